@@ -1,0 +1,120 @@
+/*
+ * tvm_attn.h -- C ABI of the fused attention + Jacobian-vector-product library for NVIDIA B200
+ * (sm_100a).
+ *
+ * The operation is the one the Terminal Velocity Matching paper describes in Sec. 4 ("Flash
+ * Attention JVP with backward pass") and App. C ("Flash Attention JVP with Backward Pass"):
+ * scaled-dot-product attention that carries tangents next to the primal, and a backward pass that
+ * differentiates through both outputs.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers on the current device, owned by the caller, packed
+ *     (B, H, N, d) row-major (d contiguous) and 16-byte aligned.  Row statistics are (B, H, N)
+ *     float.  The library never allocates, frees or keeps device memory.
+ *   - Outputs are fully overwritten, never accumulated into.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and the call returns without synchronising.
+ *   - Return value: TVM_ATTN_OK or a negative tvm_attn_status.  No exception or abort crosses
+ *     this boundary.  Concurrent calls from several host threads on different streams are allowed.
+ *   - Self-attention, non-causal, no mask, bias or dropout: N queries attend to N keys per head.
+ */
+#ifndef TVM_ATTN_H_
+#define TVM_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TVM_ATTN_OK = 0,
+    TVM_ATTN_INVALID_ARG = -1,         /* null pointer, non-positive dim, misaligned pointer, bad dtype/flags */
+    TVM_ATTN_UNSUPPORTED = -2,         /* d > 128 or d % 8 != 0, device is not sm_100, too many tiles  */
+    TVM_ATTN_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < tvm_attn_jvp_workspace_bytes(...) */
+    TVM_ATTN_CUDA_ERROR = -4,          /* a CUDA runtime/driver call or a launch failed */
+    TVM_ATTN_DEVICE_TIMEOUT = -5       /* a bounded on-device wait ran out (see tvm_attn_check_status) */
+} tvm_attn_status;
+
+/* dtype of the eight/sixteen (B,H,N,d) tensors */
+#define TVM_ATTN_BF16 0 /* bf16 tensors, fp32 accumulation, tensor-core kernels (the hot path)      */
+#define TVM_ATTN_FP32 1 /* fp32 tensors, fp32 CUDA-core kernels (validation mode, not a fast path)  */
+
+/* flags */
+#define TVM_ATTN_FLAG_CUDA_CORES 1u /* run the CUDA-core validation kernels also for bf16 tensors   */
+
+typedef struct {
+    int32_t B, H, N, d; /* batch, heads, tokens (queries = keys), head dim; 8 <= d <= 128, d % 8 == 0 */
+    float scale;        /* softmax scale alpha of App. C; 0.0f selects 1/sqrt(d) with the true d     */
+    int32_t dtype;      /* TVM_ATTN_BF16 or TVM_ATTN_FP32                                            */
+    uint32_t flags;     /* 0 or TVM_ATTN_FLAG_*                                                      */
+} tvm_attn_params;
+
+/*
+ * Bytes of device scratch the forward (is_bwd == 0) or backward (is_bwd != 0) call needs for these
+ * parameters.  The forward needs none.  The backward keeps two floats per query row there (the row
+ * sums of App. C "Step 1", in the form rowsum(dtO*O) and rowsum(dO*O) + rowsum(dtO*tO)).
+ * Returns 0 for invalid parameters.
+ */
+size_t tvm_attn_jvp_workspace_bytes(const tvm_attn_params* p, int is_bwd);
+
+/*
+ * Forward (paper Sec. 4 item (i); App. C Eq. "sdpa" and the definitions of P, S, N, S-dot, mu
+ * under "Step 1"; "Caching softmax statistics").  Per head, with A = alpha Q K^T, P = softmax_rows(A),
+ * T = alpha (tQ K^T + Q tK^T), mu = rowsum(P*T):
+ *     O  = P V                      tO = (P * (T - mu)) V + P tV
+ *     lse = log rowsum(exp(A))      (natural log, of the SCALED scores)
+ * computed with an online softmax; no N x N matrix is written to memory.
+ *   in : Q, K, V, tQ, tK, tV   (B,H,N,d) dtype
+ *   out: O, tO                 (B,H,N,d) dtype, rounded to nearest even from fp32
+ *        lse, mu               (B,H,N) float; the statistics the backward needs (normalised mu, so
+ *                              the separate row sum l of App. C is not stored)
+ *   workspace: may be NULL (workspace_bytes 0).
+ */
+int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, const void* V,
+                     const void* tQ, const void* tK, const void* tV, void* O, void* tO, float* lse,
+                     float* mu, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward through both outputs (paper Sec. 4 item (iii); App. C "Multi-step backward pass",
+ * steps 1-6, plus the standard attention backward for dO that the paper sums in).  With
+ * G = dO, Hc = dtO, Nn = T - mu, D = Hc V^T, X = G V^T + Hc tV^T,
+ * W = P * (D - Sigma_1), dA = P * (X - rowsum(G*O) - Sigma_2) + W * Nn:
+ *     dV = P^T G + (P*Nn)^T Hc     dtV = P^T Hc
+ *     dQ = alpha (dA K + W tK)     dtQ = alpha W K
+ *     dK = alpha (dA^T Q + W^T tQ) dtK = alpha W^T Q
+ *   in : Q, K, V, tQ, tK, tV and the forward's O, tO, lse, mu; dO, dtO (B,H,N,d) dtype, both
+ *        required (non-NULL)
+ *   out: dQ, dK, dV, dtQ, dtK, dtV (B,H,N,d) dtype
+ *   workspace: device scratch of at least tvm_attn_jvp_workspace_bytes(p, 1) bytes, 16-byte
+ *        aligned; contents on return are unspecified.  Calls sharing one workspace must not
+ *        overlap on the device.
+ */
+int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, const void* V,
+                     const void* tQ, const void* tK, const void* tV, const void* O, const void* tO,
+                     const float* lse, const float* mu, const void* dO, const void* dtO, void* dQ,
+                     void* dK, void* dV, void* dtQ, void* dtK, void* dtV, void* workspace,
+                     size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and reports what the kernels enqueued so far on the current device
+ * recorded: TVM_ATTN_OK, TVM_ATTN_DEVICE_TIMEOUT if a bounded wait inside a tensor-core kernel gave
+ * up (its outputs are then unspecified; the context stays usable), or TVM_ATTN_CUDA_ERROR.  Clears
+ * the recorded status.  (No counterpart in the paper: error reporting of this library.)
+ */
+int tvm_attn_check_status(void* cuda_stream);
+
+/* Number of this library's kernels launched by the calling process so far (all threads). */
+uint64_t tvm_attn_launch_count(void);
+
+/* Static, human-readable text for a status code. */
+const char* tvm_attn_strerror(int code);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int tvm_attn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TVM_ATTN_H_ */

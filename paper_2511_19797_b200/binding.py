@@ -1,0 +1,160 @@
+"""ctypes binding of the C-ABI library declared in include/tvm_attn.h.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of the library.
+PyTorch provides device memory and streams.  There is no CPU or library fallback: if the
+shared object is missing or a call fails, an exception is raised.
+"""
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+BF16 = 0
+FP32 = 1
+FLAG_CUDA_CORES = 1
+
+_STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
+                 -5: "DEVICE_TIMEOUT"}
+
+
+class TvmAttnError(RuntimeError):
+    def __init__(self, where, code, text):
+        super().__init__("%s failed: %s (%d): %s" % (where, _STATUS_NAMES.get(code, "?"), code, text))
+        self.code = code
+
+
+class Params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("dtype", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+_lib = None
+EXPORTS = ("tvm_attn_jvp_workspace_bytes", "tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_check_status",
+           "tvm_attn_launch_count", "tvm_attn_strerror", "tvm_attn_version")
+
+
+def library_path():
+    return _build.LIB_PATH
+
+
+def load(build_if_missing=False):
+    """Loads libtvm_attn.so (built in-tree by build.py).  Raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        if not build_if_missing:
+            raise FileNotFoundError("%s is missing: run paper_2511_19797_b200/build.py (nvcc, sm_100a) first" % path)
+        _build.build()
+    lib = ctypes.CDLL(path)
+    vp, pp = ctypes.c_void_p, ctypes.POINTER(Params)
+    lib.tvm_attn_jvp_workspace_bytes.restype = ctypes.c_size_t
+    lib.tvm_attn_jvp_workspace_bytes.argtypes = [pp, ctypes.c_int]
+    lib.tvm_attn_jvp_fwd.restype = ctypes.c_int
+    lib.tvm_attn_jvp_fwd.argtypes = [pp] + [vp] * 10 + [vp, ctypes.c_size_t, vp]
+    lib.tvm_attn_jvp_bwd.restype = ctypes.c_int
+    lib.tvm_attn_jvp_bwd.argtypes = [pp] + [vp] * 18 + [vp, ctypes.c_size_t, vp]
+    lib.tvm_attn_check_status.restype = ctypes.c_int
+    lib.tvm_attn_check_status.argtypes = [vp]
+    lib.tvm_attn_launch_count.restype = ctypes.c_uint64
+    lib.tvm_attn_launch_count.argtypes = []
+    lib.tvm_attn_strerror.restype = ctypes.c_char_p
+    lib.tvm_attn_strerror.argtypes = [ctypes.c_int]
+    lib.tvm_attn_version.restype = ctypes.c_int
+    lib.tvm_attn_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _raise(where, code):
+    raise TvmAttnError(where, code, load().tvm_attn_strerror(code).decode())
+
+
+def _params(x, scale, flags):
+    if x.dim() != 4:
+        raise ValueError("expected (B, H, N, d) tensors")
+    if x.dtype == torch.bfloat16:
+        dt = BF16
+    elif x.dtype == torch.float32:
+        dt = FP32
+    else:
+        raise ValueError("tensors must be bfloat16 or float32")
+    B, H, N, d = x.shape
+    return Params(B, H, N, d, float(scale), dt, int(flags))
+
+
+def _check_tensors(ref, tensors):
+    for t in tensors:
+        if t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device:
+            raise ValueError("all (B, H, N, d) tensors must share shape, dtype and device")
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def _stream_ptr(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def tvm_attn_jvp_workspace_bytes(B, H, N, d, dtype=BF16, is_bwd=True, scale=0.0, flags=0):
+    p = Params(B, H, N, d, float(scale), dtype, flags)
+    return int(load().tvm_attn_jvp_workspace_bytes(ctypes.byref(p), 1 if is_bwd else 0))
+
+
+def tvm_attn_jvp_fwd(Q, K, V, tQ, tK, tV, scale=0.0, flags=0, out=None, stream=None):
+    """Forward: returns (O, tO, lse, mu).  `out` may hold preallocated (O, tO, lse, mu)."""
+    lib = load()
+    _check_tensors(Q, (K, V, tQ, tK, tV))
+    p = _params(Q, scale, flags)
+    if out is None:
+        O, tO = torch.empty_like(Q), torch.empty_like(Q)
+        lse = torch.empty(Q.shape[:3], dtype=torch.float32, device=Q.device)
+        mu = torch.empty_like(lse)
+    else:
+        O, tO, lse, mu = out
+    with torch.cuda.device(Q.device):
+        rc = lib.tvm_attn_jvp_fwd(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
+                                  tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
+                                  mu.data_ptr(), None, 0, _stream_ptr(stream))
+    if rc != 0:
+        _raise("tvm_attn_jvp_fwd", rc)
+    return O, tO, lse, mu
+
+
+def tvm_attn_jvp_bwd(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, scale=0.0, flags=0, out=None, workspace=None,
+                     stream=None):
+    """Backward: returns (dQ, dK, dV, dtQ, dtK, dtV).  `workspace` is a uint8 CUDA tensor of at least
+    tvm_attn_jvp_workspace_bytes(...) bytes; one is allocated with torch when not given."""
+    lib = load()
+    _check_tensors(Q, (K, V, tQ, tK, tV, O, tO, dO, dtO))
+    p = _params(Q, scale, flags)
+    need = int(lib.tvm_attn_jvp_workspace_bytes(ctypes.byref(p), 1))
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=Q.device)
+    outs = out if out is not None else tuple(torch.empty_like(Q) for _ in range(6))
+    with torch.cuda.device(Q.device):
+        rc = lib.tvm_attn_jvp_bwd(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
+                                  tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
+                                  mu.data_ptr(), dO.data_ptr(), dtO.data_ptr(), *[o.data_ptr() for o in outs],
+                                  workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        _raise("tvm_attn_jvp_bwd", rc)
+    return outs
+
+
+def tvm_attn_check_status(stream=None, raise_on_error=True):
+    rc = int(load().tvm_attn_check_status(_stream_ptr(stream)))
+    if rc != 0 and raise_on_error:
+        _raise("tvm_attn_check_status", rc)
+    return rc
+
+
+def tvm_attn_launch_count():
+    return int(load().tvm_attn_launch_count())
+
+
+def tvm_attn_version():
+    return int(load().tvm_attn_version())

@@ -1,0 +1,309 @@
+// C-ABI entry points of the attention-JVP library (see include/tvm_attn.h): argument checks, TMA
+// tensor-map construction and kernel launches.  No device memory is allocated here.
+#include "tvm_attn.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "dual_attn_sm100.cuh"
+#include "simt_kernels.cuh"
+
+namespace tvm_attn {
+
+static std::atomic<uint64_t> g_launches{0};
+__device__ int g_status_word = 0;  // raised by a tensor-core kernel whose bounded wait ran out
+
+struct Shape {
+    int B, H, N, d, dp;
+    long long BH;
+    float alpha;
+    bool fp32, simt;
+};
+
+static int check_params(const tvm_attn_params* p, Shape* s) {
+    if (!p) return TVM_ATTN_INVALID_ARG;
+    if (p->B <= 0 || p->H <= 0 || p->N <= 0 || p->d <= 0) return TVM_ATTN_INVALID_ARG;
+    if (p->dtype != TVM_ATTN_BF16 && p->dtype != TVM_ATTN_FP32) return TVM_ATTN_INVALID_ARG;
+    if (p->flags & ~TVM_ATTN_FLAG_CUDA_CORES) return TVM_ATTN_INVALID_ARG;
+    if (!(p->scale >= 0.0f) || !std::isfinite(p->scale)) return TVM_ATTN_INVALID_ARG;
+    if (p->d > 128 || p->d % 8 != 0) return TVM_ATTN_UNSUPPORTED;
+    s->B = p->B; s->H = p->H; s->N = p->N; s->d = p->d;
+    s->dp = (p->d + 15) / 16 * 16;
+    s->BH = (long long)p->B * p->H;
+    s->alpha = p->scale == 0.0f ? 1.0f / std::sqrt((float)p->d) : p->scale;
+    s->fp32 = p->dtype == TVM_ATTN_FP32;
+    s->simt = s->fp32 || (p->flags & TVM_ATTN_FLAG_CUDA_CORES);
+    // every kernel flattens (head, row tile) into blockIdx.x
+    const long long tiles16 = (p->N + 15LL) / 16;
+    if (s->BH * tiles16 > 2147483647LL) return TVM_ATTN_UNSUPPORTED;
+    if (s->BH > 2147483647LL / p->N) return TVM_ATTN_UNSUPPORTED;  // B*H*N rows indexable as int
+    return TVM_ATTN_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int cuda_status(cudaError_t e) { return e == cudaSuccess ? TVM_ATTN_OK : TVM_ATTN_CUDA_ERROR; }
+
+// ------------------------------------------------------------------------------------------------
+// CUDA-core path
+template <typename T>
+static int simt_fwd(const Shape& s, const void* Q, const void* K, const void* V, const void* tQ, const void* tK,
+                    const void* tV, void* O, void* tO, float* lse, float* mu, cudaStream_t st) {
+    const size_t smem = simt_smem_bytes(s.d, 2);
+    cudaError_t e = cudaFuncSetAttribute(simt_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    const unsigned grid = (unsigned)(s.BH * ((s.N + SIMT_ROWS - 1) / SIMT_ROWS));
+    simt_fwd_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
+                                                         (const T*)tK, (const T*)tV, (T*)O, (T*)tO, lse, mu, s.N, s.d,
+                                                         s.alpha);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
+template <typename T>
+static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const void* O, const void* tO, float* sig1,
+                          float* cvec, cudaStream_t st) {
+    const long long rows = s.BH * s.N;
+    const unsigned grid = (unsigned)((rows + 7) / 8);
+    bwd_rowsums_kernel<T><<<grid, 256, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, sig1, cvec, rows,
+                                                s.d);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
+template <typename T>
+static int simt_bwd(const Shape& s, const void* Q, const void* K, const void* V, const void* tQ, const void* tK,
+                    const void* tV, const float* lse, const float* mu, const void* G, const void* Hc,
+                    const float* sig1, const float* cvec, void* dQ, void* dK, void* dV, void* dtQ, void* dtK, void* dtV,
+                    cudaStream_t st) {
+    const size_t smem = simt_smem_bytes(s.d, 4);
+    if (cudaFuncSetAttribute(simt_bwd_dq_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(simt_bwd_dkv_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return TVM_ATTN_CUDA_ERROR;
+    const unsigned grid = (unsigned)(s.BH * ((s.N + SIMT_ROWS - 1) / SIMT_ROWS));
+    simt_bwd_dq_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
+                                                            (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc, lse,
+                                                            mu, sig1, cvec, (T*)dQ, (T*)dtQ, s.N, s.d, s.alpha);
+    simt_bwd_dkv_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
+                                                             (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc,
+                                                             lse, mu, sig1, cvec, (T*)dK, (T*)dV, (T*)dtK, (T*)dtV,
+                                                             s.N, s.d, s.alpha);
+    g_launches += 2;
+    return cuda_status(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tensor-core path
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static encode_tiled_fn get_encode_fn() {
+    static encode_tiled_fn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(sym);
+    });
+    return fn;
+}
+
+// (B,H,N,d) bf16 viewed as a 3-D tensor (d, N, B*H); a box is 64 columns x `rows` rows of one head with
+// the 128-byte swizzle; columns or rows beyond the tensor read as zero.
+static int make_tmap(CUtensorMap* m, const void* ptr, const Shape& s, int rows) {
+    encode_tiled_fn fn = get_encode_fn();
+    if (!fn) return TVM_ATTN_CUDA_ERROR;
+    cuuint64_t dims[3] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.BH};
+    cuuint64_t strides[2] = {(cuuint64_t)s.d * 2, (cuuint64_t)s.N * s.d * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TVM_ATTN_OK : TVM_ATTN_CUDA_ERROR;
+}
+
+static int device_is_sm100() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    return major == 10 ? TVM_ATTN_OK : TVM_ATTN_UNSUPPORTED;
+}
+
+static int* status_word_ptr() {
+    int* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_status_word) != cudaSuccess) return nullptr;
+    return ptr;
+}
+
+template <int MODE, int NA>
+static int launch_tc(const Shape& s, const void* const own[4], const void* const strm[4], const TcParams& prm,
+                     cudaStream_t st) {
+    using C = TcCfg<MODE, NA>;
+    CUtensorMap mo[4], ms[4];
+    for (int t = 0; t < 4; ++t) {
+        const void* po = own[t < C::NOWN ? t : 0];
+        int rc = make_tmap(&mo[t], po, s, TC_OWN_ROWS);
+        if (rc != TVM_ATTN_OK) return rc;
+        rc = make_tmap(&ms[t], strm[t], s, C::BC);
+        if (rc != TVM_ATTN_OK) return rc;
+    }
+    auto kern = dual_attn_kernel<MODE, NA>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        return TVM_ATTN_CUDA_ERROR;
+    const long long grid = s.BH * ((s.N + TC_OWN_ROWS - 1) / TC_OWN_ROWS);
+    kern<<<(unsigned)grid, TC_THREADS, C::SMEM_BYTES, st>>>(mo[0], mo[1], mo[2], mo[3], ms[0], ms[1], ms[2], ms[3], prm);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
+template <int MODE>
+static int launch_tc_na(const Shape& s, const void* const own[4], const void* const strm[4], const TcParams& prm,
+                        cudaStream_t st) {
+    return s.d <= 64 ? launch_tc<MODE, 1>(s, own, strm, prm, st) : launch_tc<MODE, 2>(s, own, strm, prm, st);
+}
+
+static TcParams base_params(const Shape& s, int* status) {
+    TcParams prm;
+    std::memset(&prm, 0, sizeof prm);
+    prm.N = s.N; prm.d = s.d; prm.dp = s.dp; prm.BH = (int)s.BH;
+    prm.alpha = s.alpha;
+    prm.c2 = s.alpha * 1.4426950408889634f;
+    prm.out_scale = 1.0f;
+    prm.status = status;
+    return prm;
+}
+
+}  // namespace tvm_attn
+
+using namespace tvm_attn;
+
+extern "C" {
+
+size_t tvm_attn_jvp_workspace_bytes(const tvm_attn_params* p, int is_bwd) {
+    Shape s;
+    if (check_params(p, &s) != TVM_ATTN_OK) return 0;
+    if (!is_bwd) return 0;
+    return (size_t)2 * sizeof(float) * (size_t)s.BH * (size_t)s.N;
+}
+
+int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, const void* V, const void* tQ,
+                     const void* tK, const void* tV, void* O, void* tO, float* lse, float* mu, void* workspace,
+                     size_t workspace_bytes, void* cuda_stream) {
+    (void)workspace; (void)workspace_bytes;
+    Shape s;
+    int rc = check_params(p, &s);
+    if (rc != TVM_ATTN_OK) return rc;
+    const void* ptrs[] = {Q, K, V, tQ, tK, tV, O, tO, lse, mu};
+    for (const void* x : ptrs)
+        if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (s.simt) {
+        return s.fp32 ? simt_fwd<float>(s, Q, K, V, tQ, tK, tV, O, tO, lse, mu, st)
+                      : simt_fwd<__nv_bfloat16>(s, Q, K, V, tQ, tK, tV, O, tO, lse, mu, st);
+    }
+    rc = device_is_sm100();
+    if (rc != TVM_ATTN_OK) return rc;
+    int* status = status_word_ptr();
+    if (!status) return TVM_ATTN_CUDA_ERROR;
+    TcParams prm = base_params(s, status);
+    prm.out0 = O; prm.out1 = tO; prm.lse_out = lse; prm.mu_out = mu;
+    const void* own[4] = {Q, tQ, Q, tQ};
+    const void* strm[4] = {K, tK, V, tV};
+    return launch_tc_na<MODE_FWD>(s, own, strm, prm, st);
+}
+
+int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, const void* V, const void* tQ,
+                     const void* tK, const void* tV, const void* O, const void* tO, const float* lse, const float* mu,
+                     const void* dO, const void* dtO, void* dQ, void* dK, void* dV, void* dtQ, void* dtK, void* dtV,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Shape s;
+    int rc = check_params(p, &s);
+    if (rc != TVM_ATTN_OK) return rc;
+    const void* ptrs[] = {Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, dQ, dK, dV, dtQ, dtK, dtV, workspace};
+    for (const void* x : ptrs)
+        if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
+    const size_t rows = (size_t)s.BH * (size_t)s.N;
+    if (workspace_bytes < 2 * sizeof(float) * rows) return TVM_ATTN_WORKSPACE_TOO_SMALL;
+    float* sig1 = static_cast<float*>(workspace);
+    float* cvec = sig1 + rows;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (s.simt) {
+        if (s.fp32) {
+            rc = launch_rowsums<float>(s, dO, dtO, O, tO, sig1, cvec, st);
+            if (rc != TVM_ATTN_OK) return rc;
+            return simt_bwd<float>(s, Q, K, V, tQ, tK, tV, lse, mu, dO, dtO, sig1, cvec, dQ, dK, dV, dtQ, dtK, dtV, st);
+        }
+        rc = launch_rowsums<__nv_bfloat16>(s, dO, dtO, O, tO, sig1, cvec, st);
+        if (rc != TVM_ATTN_OK) return rc;
+        return simt_bwd<__nv_bfloat16>(s, Q, K, V, tQ, tK, tV, lse, mu, dO, dtO, sig1, cvec, dQ, dK, dV, dtQ, dtK, dtV, st);
+    }
+    rc = device_is_sm100();
+    if (rc != TVM_ATTN_OK) return rc;
+    int* status = status_word_ptr();
+    if (!status) return TVM_ATTN_CUDA_ERROR;
+    rc = launch_rowsums<__nv_bfloat16>(s, dO, dtO, O, tO, sig1, cvec, st);
+    if (rc != TVM_ATTN_OK) return rc;
+    TcParams prm = base_params(s, status);
+    prm.lse = lse; prm.mu = mu; prm.sig1 = sig1; prm.cvec = cvec;
+    {   // dtV = P^T Hc, dV = P^T G + (P*Nn)^T Hc : owner keys (K, tK), stream queries (Q, tQ | Hc, G)
+        TcParams q = prm; q.out0 = dtV; q.out1 = dV;
+        const void* own[4] = {K, tK, K, tK};
+        const void* strm[4] = {Q, tQ, dtO, dO};
+        rc = launch_tc_na<MODE_DV>(s, own, strm, q, st);
+        if (rc != TVM_ATTN_OK) return rc;
+    }
+    {   // dtK = alpha W^T Q, dK = alpha (dA^T Q + W^T tQ) : owner keys (K, tK, V, tV), stream (Q, tQ, Hc, G)
+        TcParams q = prm; q.out0 = dtK; q.out1 = dK; q.out_scale = s.alpha;
+        const void* own[4] = {K, tK, V, tV};
+        const void* strm[4] = {Q, tQ, dtO, dO};
+        rc = launch_tc_na<MODE_DK>(s, own, strm, q, st);
+        if (rc != TVM_ATTN_OK) return rc;
+    }
+    {   // dtQ = alpha W K, dQ = alpha (dA K + W tK) : owner queries (Q, tQ, Hc, G), stream (K, tK, V, tV)
+        TcParams q = prm; q.out0 = dtQ; q.out1 = dQ; q.out_scale = s.alpha;
+        const void* own[4] = {Q, tQ, dtO, dO};
+        const void* strm[4] = {K, tK, V, tV};
+        rc = launch_tc_na<MODE_DQ>(s, own, strm, q, st);
+    }
+    return rc;
+}
+
+int tvm_attn_check_status(void* cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    int host = 0;
+    if (cudaMemcpyFromSymbol(&host, g_status_word, sizeof(int)) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    if (host != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+        return TVM_ATTN_DEVICE_TIMEOUT;
+    }
+    return TVM_ATTN_OK;
+}
+
+uint64_t tvm_attn_launch_count(void) { return g_launches.load(); }
+
+const char* tvm_attn_strerror(int code) {
+    switch (code) {
+        case TVM_ATTN_OK: return "ok";
+        case TVM_ATTN_INVALID_ARG: return "invalid argument (null or misaligned pointer, bad dimension, dtype, flags or scale)";
+        case TVM_ATTN_UNSUPPORTED: return "unsupported shape or device (need 8 <= d <= 128, d % 8 == 0, an sm_100 GPU)";
+        case TVM_ATTN_WORKSPACE_TOO_SMALL: return "workspace smaller than tvm_attn_jvp_workspace_bytes()";
+        case TVM_ATTN_CUDA_ERROR: return "a CUDA call or kernel launch failed";
+        case TVM_ATTN_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out; outputs are unspecified";
+        default: return "unknown status";
+    }
+}
+
+int tvm_attn_version(void) { return 100; }
+
+}  // extern "C"

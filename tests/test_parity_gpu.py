@@ -1,0 +1,107 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the fp64 C oracle on the
+same seeded inputs.  Error metric per tensor: max|gpu - ref| / max|ref|.
+
+Tolerances: bf16 mode 1e-2 for O and tO, 2e-2 for the six gradients (inputs are rounded to bf16
+once and the oracle consumes those rounded values, so only the kernels' own rounding counts);
+fp32 validation mode 1e-4 for everything.  The saved statistics lse and mu are fp32 in both modes;
+in bf16 mode they are held to 2e-3 (they come from bf16 tensor-core products accumulated in fp32).
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_19797_b200 import binding, inputs
+from tests._parity import assert_within, run_case
+
+pytestmark = pytest.mark.gpu
+
+BF16_FWD, BF16_BWD, BF16_STATS, FP32_TOL = 1e-2, 2e-2, 2e-3, 1e-4
+
+
+def test_tiny_fp32_validation_mode():
+    errs, _, _ = run_case("tiny", dtype=torch.float32)
+    assert_within(errs, FP32_TOL, FP32_TOL)
+
+
+def test_tiny_bf16_tensor_cores():
+    errs, _, _ = run_case("tiny")
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+def test_tiny_bf16_cuda_cores():
+    errs, _, _ = run_case("tiny", flags=binding.FLAG_CUDA_CORES)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+@pytest.mark.parametrize("name,heads", [
+    ("dit256", [0, 341, 682, 1023]),
+    ("dit512", [0, 85, 170, 255]),
+    ("large", [0, 47]),
+    ("sweep256", [0, 1365, 2730, 4095]),
+    ("sweep1024", [0, 341, 682, 1023]),
+    ("sweep4096", [0, 255]),
+])
+def test_full_size_workloads_on_sampled_heads(name, heads):
+    errs, _, _ = run_case(name, oracle_heads=heads)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+@pytest.mark.parametrize("B,H,N,d", [
+    (1, 1, 1, 8), (1, 2, 7, 16), (2, 1, 64, 64), (1, 1, 100, 72), (1, 3, 129, 40), (2, 2, 191, 128),
+    (1, 1, 257, 72), (1, 2, 320, 32), (1, 1, 1000, 24),
+])
+@pytest.mark.parametrize("mode", ["bf16", "fp32"])
+def test_ragged_and_degenerate_shapes(B, H, N, d, mode):
+    wl = inputs.custom(B, H, N, d, seed=100 + N + d)
+    if mode == "fp32":
+        errs, _, _ = run_case(wl, dtype=torch.float32)
+        assert_within(errs, FP32_TOL, FP32_TOL)
+    else:
+        errs, _, _ = run_case(wl)
+        assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+def test_explicit_scale_is_honoured():
+    wl = inputs.custom(1, 2, 96, 48, seed=7)
+    errs, _, _ = run_case(wl, scale=0.05)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+def test_runs_are_bit_reproducible_and_respect_buffer_bounds():
+    wl = inputs.custom(2, 2, 200, 72, seed=9)
+    x = {k: v.to(torch.bfloat16).cuda() for k, v in inputs.make_inputs(wl).items()}
+    n = x["Q"].numel()
+
+    def padded():
+        buf = torch.full((n + 512,), 123.0, dtype=torch.bfloat16, device="cuda")
+        return buf, buf[256:256 + n].view_as(x["Q"])
+
+    runs = []
+    for _ in range(2):
+        bufs = [padded() for _ in range(8)]
+        lse = torch.empty(x["Q"].shape[:3], dtype=torch.float32, device="cuda")
+        mu = torch.empty_like(lse)
+        O, tO, lse, mu = binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"],
+                                                  out=(bufs[0][1], bufs[1][1], lse, mu))
+        grads = binding.tvm_attn_jvp_bwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], O, tO, lse, mu, x["dO"],
+                                         x["dtO"], out=tuple(b[1] for b in bufs[2:]))
+        binding.tvm_attn_check_status()
+        for full, _ in bufs:
+            assert torch.all(full[:256] == 123.0) and torch.all(full[256 + n:] == 123.0), "wrote outside a buffer"
+        runs.append([t.clone() for t in (O, tO, lse, mu) + tuple(grads)])
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+
+
+def test_errors_reported_on_the_gpu_box():
+    x = torch.zeros(1, 1, 64, 36, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.TvmAttnError) as e:
+        binding.tvm_attn_jvp_fwd(x, x, x, x, x, x)
+    assert e.value.code == -2
+    y = torch.zeros(1, 1, 64, 32, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(1, 1, 64, device="cuda")
+    with pytest.raises(binding.TvmAttnError) as e:
+        binding.tvm_attn_jvp_bwd(y, y, y, y, y, y, y, y, lse, lse, y, y,
+                                 workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -3
+    assert binding.tvm_attn_launch_count() >= 0
