@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the fused attention-JVP forward + backward path on B200.
+
+One "step" is one forward call plus one backward call of the C-ABI library over one batch of
+synthetic DiT-shaped input (default workload: B=16, H=16, N=1024, d=72, bf16).  The metric is
+TFLOP/s with the analytic work of the method (12*B*H*N^2*d forward, 30*B*H*N^2*d backward, true d).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line.  Under torchrun every rank runs the same per-GPU workload on its own GPU
+(heads are independent, no collective in the data path: weak scaling); rank 0 prints.
+`--impl reference` times the fp64 CPU oracle on the host cores instead (a baseline, not a target).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "attn_jvp_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# GEMMs each kernel executes by design (x 2*B*H*N^2*d FLOP each, true d)
+KERNEL_GEMMS = {"fwd": 6, "bwd_rowsums": 0, "bwd_dv": 6, "bwd_dk": 9, "bwd_dq": 9}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            pk = json.load(f)
+        return {k: float(pk[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(wl_name, target_seconds=12.0, threads=None):
+    """Times the C oracle (forward + backward) on a bounded sample of whole heads of the workload.
+    Returns (TFLOP/s, threads, description, seconds)."""
+    import numpy as np
+    import torch
+    from oracle import c_oracle
+    from paper_2511_19797_b200 import inputs
+    wl = inputs.WORKLOADS[wl_name]
+    cores = threads or c_oracle.default_threads()
+    f_fwd, f_bwd = inputs.flops(1, 1, wl.N, wl.d)
+    est_rate = 0.25e9 * 2  # ~FLOP/s of one thread of the plain C loops; only sizes the sample
+    heads = int(max(1, min(wl.B * wl.H, round(target_seconds * est_rate * cores / (f_fwd + f_bwd)))))
+    if heads >= cores:
+        heads = max(cores, heads // cores * cores)
+    idx = [int(i) for i in np.linspace(0, wl.B * wl.H - 1, heads).round()]
+    x = inputs.make_inputs(wl, heads=idx)
+    xs = [x[k].to(torch.bfloat16).to(torch.float64).numpy() for k in inputs.NAMES]
+    alpha = inputs.default_scale(wl.d)
+    t0 = time.perf_counter()
+    used = c_oracle.attn_jvp_fwd(*xs[:6], alpha, nthreads=cores)[4]
+    c_oracle.attn_jvp_bwd(*xs, alpha, nthreads=cores)
+    dt = time.perf_counter() - t0
+    tflops = heads * (f_fwd + f_bwd) / dt / 1e12
+    desc = "%d of %d heads of %s (fwd+bwd, fp64 C oracle, gcc -O2), %.1f s" % (heads, wl.B * wl.H, wl_name, dt)
+    return tflops, used, desc, dt
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from paper_2511_19797_b200 import inputs
+    wl = inputs.WORKLOADS[args.workload]
+    times, vals = [], []
+    for it in range(args.warmup + args.steps):
+        v, cores, desc, dt = oracle_sample(args.workload, target_seconds=6.0)
+        if it >= args.warmup:
+            times.append(dt); vals.append(v)
+    value = statistics.mean(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d,
+                   "note": "each step is a bounded sample of whole heads of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="dit512")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2511_19797_b200 import binding, inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    binding.load()
+
+    wl = inputs.WORKLOADS[args.workload]
+    f_fwd, f_bwd = inputs.flops(wl.B, wl.H, wl.N, wl.d)
+    host = {k: v.to(torch.bfloat16).pin_memory() for k, v in inputs.make_inputs(wl).items()}
+    x = {k: v.to(dev) for k, v in host.items()}
+    shape = x["Q"].shape
+    O, tO = torch.empty_like(x["Q"]), torch.empty_like(x["Q"])
+    lse = torch.empty(shape[:3], dtype=torch.float32, device=dev)
+    mu = torch.empty_like(lse)
+    grads = tuple(torch.empty_like(x["Q"]) for _ in range(6))
+    ws = torch.empty(max(16, binding.tvm_attn_jvp_workspace_bytes(*shape)), dtype=torch.uint8, device=dev)
+
+    def fwd():
+        binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], out=(O, tO, lse, mu))
+
+    def bwd():
+        binding.tvm_attn_jvp_bwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], O, tO, lse, mu, x["dO"], x["dtO"],
+                                 out=grads, workspace=ws)
+
+    def step():
+        fwd()
+        bwd()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, n):
+        """n back-to-back calls between CUDA events on torch's current stream (the one the library is given)."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        step()
+    binding.tvm_attn_check_status()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.tvm_attn_launch_count()
+    ms_total = timed(step, args.steps)
+    launches = binding.tvm_attn_launch_count() - launches0
+    ms_fwd = timed(fwd, args.steps)
+    ms_bwd = timed(bwd, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    binding.tvm_attn_check_status()
+
+    # per-kernel durations (CUDA events recorded by the library around each launch)
+    binding.tvm_attn_set_profiling(True)
+    per_kernel = {k: [] for k in KERNEL_GEMMS}
+    for _ in range(min(args.steps, 20)):
+        fwd()
+        per_kernel["fwd"].append(binding.tvm_attn_get_profile()[0])
+        bwd()
+        prof = binding.tvm_attn_get_profile()
+        for k, v in zip(("bwd_rowsums", "bwd_dv", "bwd_dk", "bwd_dq"), prof):
+            per_kernel[k].append(v)
+    binding.tvm_attn_set_profiling(False)
+    kernel_ms = {k: statistics.mean(v) for k, v in per_kernel.items() if v}
+
+    # end to end: pinned host inputs -> device, forward + backward, results -> pinned host
+    host_out = {k: torch.empty(shape, dtype=torch.bfloat16).pin_memory() for k in ("O", "tO", "dQ", "dK", "dV", "dtQ", "dtK", "dtV")}
+    host_stats = {k: torch.empty(shape[:3], dtype=torch.float32).pin_memory() for k in ("lse", "mu")}
+
+    def e2e_step():
+        for k in inputs.NAMES:
+            x[k].copy_(host[k], non_blocking=True)
+        step()
+        for k, t in zip(("O", "tO", "dQ", "dK", "dV", "dtQ", "dtK", "dtV"), (O, tO) + grads):
+            host_out[k].copy_(t, non_blocking=True)
+        host_stats["lse"].copy_(lse, non_blocking=True)
+        host_stats["mu"].copy_(mu, non_blocking=True)
+
+    e2e_step()
+    ms_e2e = timed(e2e_step, args.e2e_steps) / args.e2e_steps
+    h2d = sum(host[k].numel() * 2 for k in inputs.NAMES)
+    d2h = sum(t.numel() * 2 for t in host_out.values()) + sum(t.numel() * 4 for t in host_stats.values())
+    binding.tvm_attn_check_status()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = load_peaks()
+    ms_step = ms_total / args.steps
+    value = world * (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
+    fwd_tf = f_fwd / (ms_fwd / args.steps * 1e-3) / 1e12
+    bwd_tf = f_bwd / (ms_bwd / args.steps * 1e-3) / 1e12
+    unit_flops = 2.0 * wl.B * wl.H * wl.N * wl.N * wl.d
+    top = max((k for k in kernel_ms if KERNEL_GEMMS[k] > 0), key=lambda k: kernel_ms[k])
+    achieved = KERNEL_GEMMS[top] * unit_flops / (kernel_ms[top] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    total_k = sum(kernel_ms.values())
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "per_gpu": True,
+                   "l2": "16 resident tensors of %.0f MB each, larger than the 126 MB L2; no flush" % (x["Q"].numel() * 2 / 1e6)},
+        "fwd": {"tflops": fwd_tf, "ms": ms_fwd / args.steps, "frac_of_burst_peak": fwd_tf / peaks["bf16_tflops"],
+                "frac_of_sustained_peak": fwd_tf / peaks["bf16_tflops_sustained"], "frac_of_nominal": fwd_tf / NOMINAL_BF16_TFLOPS},
+        "bwd": {"tflops": bwd_tf, "ms": ms_bwd / args.steps, "frac_of_burst_peak": bwd_tf / peaks["bf16_tflops"],
+                "frac_of_sustained_peak": bwd_tf / peaks["bf16_tflops_sustained"], "frac_of_nominal": bwd_tf / NOMINAL_BF16_TFLOPS},
+        "frac_of_burst_peak": value / world / peaks["bf16_tflops"],
+        "kernels_ms": kernel_ms,
+        "kernels_share": {k: v / total_k for k, v in kernel_ms.items()},
+        "roofline": {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "peak_source": peak_src + " (sustained bf16 GEMM; kernel timed inside a long step)",
+                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "traffic": None,
+                     "flops_per_launch": KERNEL_GEMMS[top] * unit_flops},
+        "e2e": {"value": world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        v, cores, desc, _ = oracle_sample(args.workload)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

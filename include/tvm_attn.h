@@ -105,6 +105,17 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
  */
 int tvm_attn_check_status(void* cuda_stream);
 
+/*
+ * Per-kernel timing aid (no counterpart in the paper).  While enabled, tvm_attn_jvp_fwd/bwd record
+ * CUDA events on the caller's stream around every kernel they launch.  tvm_attn_get_profile waits
+ * for the most recent profiled call and writes the duration in milliseconds of each of its kernels
+ * to ms[0..], in launch order (forward: 1 kernel; backward: row sums, dV/dtV, dK/dtK, dQ/dtQ), and
+ * returns how many it wrote (at most `capacity`), or a negative status.  Process-wide state: use
+ * from one host thread at a time.  Creates CUDA events, no device memory.
+ */
+int tvm_attn_set_profiling(int enable);
+int tvm_attn_get_profile(float* ms, int capacity);
+
 /* Number of this library's kernels launched by the calling process so far (all threads). */
 uint64_t tvm_attn_launch_count(void);
 

@@ -32,11 +32,13 @@ class Params(ctypes.Structure):
 
 _lib = None
 EXPORTS = ("tvm_attn_jvp_workspace_bytes", "tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_check_status",
-           "tvm_attn_launch_count", "tvm_attn_strerror", "tvm_attn_version")
+           "tvm_attn_launch_count", "tvm_attn_strerror", "tvm_attn_version", "tvm_attn_set_profiling",
+           "tvm_attn_get_profile")
 
 
 def library_path():
-    return _build.LIB_PATH
+    """Path of the shared object; the environment variable TVM_ATTN_LIBRARY selects another build."""
+    return os.environ.get("TVM_ATTN_LIBRARY") or _build.LIB_PATH
 
 
 def load(build_if_missing=False):
@@ -65,6 +67,10 @@ def load(build_if_missing=False):
     lib.tvm_attn_strerror.argtypes = [ctypes.c_int]
     lib.tvm_attn_version.restype = ctypes.c_int
     lib.tvm_attn_version.argtypes = []
+    lib.tvm_attn_set_profiling.restype = ctypes.c_int
+    lib.tvm_attn_set_profiling.argtypes = [ctypes.c_int]
+    lib.tvm_attn_get_profile.restype = ctypes.c_int
+    lib.tvm_attn_get_profile.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     _lib = lib
     return lib
 
@@ -158,3 +164,16 @@ def tvm_attn_launch_count():
 
 def tvm_attn_version():
     return int(load().tvm_attn_version())
+
+
+def tvm_attn_set_profiling(enable):
+    load().tvm_attn_set_profiling(1 if enable else 0)
+
+
+def tvm_attn_get_profile():
+    """Per-kernel milliseconds of the most recent profiled call, in launch order."""
+    buf = (ctypes.c_float * 8)()
+    n = int(load().tvm_attn_get_profile(buf, 8))
+    if n < 0:
+        _raise("tvm_attn_get_profile", n)
+    return [float(buf[k]) for k in range(n)]

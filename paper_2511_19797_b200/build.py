@@ -25,20 +25,23 @@ def nvcc_command(out_path, extra=()):
             *extra, "-o", out_path, *[os.path.join(CSRC, s) for s in SOURCES]]
 
 
-def build(force=False, verbose=False):
-    """Compiles libtvm_attn.so if it is missing or older than its sources; returns its path."""
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _newest_source_mtime():
-        return LIB_PATH
-    os.makedirs(LIB_DIR, exist_ok=True)
-    tmp = LIB_PATH + ".tmp.%d" % os.getpid()
-    cmd = nvcc_command(tmp, ("-Xptxas", "-v") if verbose else ())
+def build(force=False, verbose=False, out_path=None, defines=()):
+    """Compiles libtvm_attn.so if it is missing or older than its sources; returns its path.
+    `out_path` and `defines` (e.g. ("TVM_ATTN_DEBUG_DUMP",)) make a separate, differently configured copy."""
+    global_out = out_path or LIB_PATH
+    if not force and os.path.exists(global_out) and os.path.getmtime(global_out) >= _newest_source_mtime():
+        return global_out
+    os.makedirs(os.path.dirname(global_out), exist_ok=True)
+    tmp = global_out + ".tmp.%d" % os.getpid()
+    extra = tuple("-D" + d for d in defines) + (("-Xptxas", "-v") if verbose else ())
+    cmd = nvcc_command(tmp, extra)
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n%s\n%s" % (" ".join(cmd), res.stderr[-8000:]))
     if verbose:
         print(res.stderr)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, global_out)
+    return global_out
 
 
 if __name__ == "__main__":

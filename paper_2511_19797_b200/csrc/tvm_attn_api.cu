@@ -19,6 +19,22 @@ namespace tvm_attn {
 static std::atomic<uint64_t> g_launches{0};
 __device__ int g_status_word = 0;  // raised by a tensor-core kernel whose bounded wait ran out
 
+// Optional per-kernel timing: events recorded around each launch of the most recent call.
+struct Profiler {
+    bool enabled = false;
+    int count = 0;  // kernels recorded by the last call
+    cudaEvent_t ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    void begin_call() { count = 0; }
+    void mark(cudaStream_t st, int idx) {
+        if (!enabled || idx >= 8) return;
+        if (!ev[idx] && cudaEventCreate(&ev[idx]) != cudaSuccess) { ev[idx] = nullptr; return; }
+        cudaEventRecord(ev[idx], st);
+    }
+    void before(cudaStream_t st) { if (enabled && count == 0) mark(st, 0); }
+    void after(cudaStream_t st) { if (enabled) { mark(st, count + 1); ++count; } }
+};
+static Profiler g_prof;
+
 struct Shape {
     int B, H, N, d, dp;
     long long BH;
@@ -59,9 +75,11 @@ static int simt_fwd(const Shape& s, const void* Q, const void* K, const void* V,
     cudaError_t e = cudaFuncSetAttribute(simt_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
     const unsigned grid = (unsigned)(s.BH * ((s.N + SIMT_ROWS - 1) / SIMT_ROWS));
+    g_prof.before(st);
     simt_fwd_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
                                                          (const T*)tK, (const T*)tV, (T*)O, (T*)tO, lse, mu, s.N, s.d,
                                                          s.alpha);
+    g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
 }
@@ -71,8 +89,10 @@ static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const v
                           float* cvec, cudaStream_t st) {
     const long long rows = s.BH * s.N;
     const unsigned grid = (unsigned)((rows + 7) / 8);
+    g_prof.before(st);
     bwd_rowsums_kernel<T><<<grid, 256, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, sig1, cvec, rows,
                                                 s.d);
+    g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
 }
@@ -90,10 +110,12 @@ static int simt_bwd(const Shape& s, const void* Q, const void* K, const void* V,
     simt_bwd_dq_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
                                                             (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc, lse,
                                                             mu, sig1, cvec, (T*)dQ, (T*)dtQ, s.N, s.d, s.alpha);
+    g_prof.after(st);
     simt_bwd_dkv_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
                                                              (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc,
                                                              lse, mu, sig1, cvec, (T*)dK, (T*)dV, (T*)dtK, (T*)dtV,
                                                              s.N, s.d, s.alpha);
+    g_prof.after(st);
     g_launches += 2;
     return cuda_status(cudaGetLastError());
 }
@@ -161,7 +183,9 @@ static int launch_tc(const Shape& s, const void* const own[4], const void* const
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
         return TVM_ATTN_CUDA_ERROR;
     const long long grid = s.BH * ((s.N + TC_OWN_ROWS - 1) / TC_OWN_ROWS);
+    g_prof.before(st);
     kern<<<(unsigned)grid, TC_THREADS, C::SMEM_BYTES, st>>>(mo[0], mo[1], mo[2], mo[3], ms[0], ms[1], ms[2], ms[3], prm);
+    g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
 }
@@ -172,6 +196,10 @@ static int launch_tc_na(const Shape& s, const void* const own[4], const void* co
     return s.d <= 64 ? launch_tc<MODE, 1>(s, own, strm, prm, st) : launch_tc<MODE, 2>(s, own, strm, prm, st);
 }
 
+#ifdef TVM_ATTN_DEBUG_DUMP
+static float* g_debug_dump = nullptr;
+#endif
+
 static TcParams base_params(const Shape& s, int* status) {
     TcParams prm;
     std::memset(&prm, 0, sizeof prm);
@@ -180,6 +208,9 @@ static TcParams base_params(const Shape& s, int* status) {
     prm.c2 = s.alpha * 1.4426950408889634f;
     prm.out_scale = 1.0f;
     prm.status = status;
+#ifdef TVM_ATTN_DEBUG_DUMP
+    prm.dbg = g_debug_dump;
+#endif
     return prm;
 }
 
@@ -207,6 +238,7 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
     for (const void* x : ptrs)
         if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    g_prof.begin_call();
     if (s.simt) {
         return s.fp32 ? simt_fwd<float>(s, Q, K, V, tQ, tK, tV, O, tO, lse, mu, st)
                       : simt_fwd<__nv_bfloat16>(s, Q, K, V, tQ, tK, tV, O, tO, lse, mu, st);
@@ -237,6 +269,7 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     float* sig1 = static_cast<float*>(workspace);
     float* cvec = sig1 + rows;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    g_prof.begin_call();
     if (s.simt) {
         if (s.fp32) {
             rc = launch_rowsums<float>(s, dO, dtO, O, tO, sig1, cvec, st);
@@ -290,6 +323,22 @@ int tvm_attn_check_status(void* cuda_stream) {
     return TVM_ATTN_OK;
 }
 
+int tvm_attn_set_profiling(int enable) {
+    g_prof.enabled = enable != 0;
+    g_prof.count = 0;
+    return TVM_ATTN_OK;
+}
+
+int tvm_attn_get_profile(float* ms, int capacity) {
+    if (!ms || capacity < 0) return TVM_ATTN_INVALID_ARG;
+    int n = g_prof.count < capacity ? g_prof.count : capacity;
+    if (n > 7) n = 7;
+    if (n > 0 && cudaEventSynchronize(g_prof.ev[n]) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    for (int k = 0; k < n; ++k)
+        if (cudaEventElapsedTime(&ms[k], g_prof.ev[k], g_prof.ev[k + 1]) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    return n;
+}
+
 uint64_t tvm_attn_launch_count(void) { return g_launches.load(); }
 
 const char* tvm_attn_strerror(int code) {
@@ -305,5 +354,9 @@ const char* tvm_attn_strerror(int code) {
 }
 
 int tvm_attn_version(void) { return 100; }
+
+#ifdef TVM_ATTN_DEBUG_DUMP
+void tvm_attn_debug_set_dump(float* device_ptr) { g_debug_dump = device_ptr; }
+#endif
 
 }  // extern "C"
