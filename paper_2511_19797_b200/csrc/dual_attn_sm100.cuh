@@ -45,6 +45,7 @@ constexpr int TC_OWN_ROWS = 128;
 constexpr int TC_STATS_STAGES = 4;
 constexpr uint64_t TC_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;  // 0.2 s per wait
 constexpr float TC_RESCALE_THRESHOLD = 8.0f;  // log2 units: accumulators are rescaled only past this
+constexpr float TC_CENTER_DELTA = 3.0f;       // the centre of the tangent weights moves only past this
 
 struct TcParams {
     int N, d, dp, BH;
@@ -89,13 +90,71 @@ struct TcCfg {
     static constexpr int B_XCHG = B_STEMPTY + TC_STATS_STAGES;
     static constexpr int NBARS = B_XCHG + 4;
     static constexpr int MISC_BYTES = 8 * 64 /*barriers*/ + 64 /*tmem ptr, abort*/ +
-                                      TC_STATS_STAGES * 4 * 64 * 4 /*stats*/ + 2 * 2 * 128 * 4 /*xchg*/;
+                                      TC_STATS_STAGES * 4 * 64 * 4 /*stats*/ + 2 * 2 * 2 * 128 * 4 /*xchg*/;
     static constexpr int SMEM_BYTES = TILE_BYTES + MISC_BYTES + 1024 /*alignment slack*/;
     static_assert(NBARS <= 64, "barrier table too small");
     // TMEM columns
     static constexpr int COL_ACC0 = 0, COL_ACC1 = 128, COL_SCORE = 256, SCORE_BUF_COLS = 2 * NPAIR * BC;
     static_assert(COL_SCORE + 2 * SCORE_BUF_COLS <= 512, "TMEM over-subscribed");
 };
+
+
+// ---- MMA issue helpers.  One thread issues every tcgen05.mma of a CTA, so the instruction count per
+// MMA matters: descriptors are built once per tile and advanced by compile-time offsets.
+
+// One GEMM  D[128 x ROWS_B] (+)= A[128 x 16*KS] * B[ROWS_B x 16*KS]^T  from K-major tiles whose
+// 64-column atoms are `rows * 128` bytes apart; k-step kk lives 32*(kk%4) bytes into atom kk/4.
+template <int KS, int ROWS_B>
+__device__ __forceinline__ void issue_kmajor_gemm(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, bool accumulate) {
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+        const uint64_t off_a = (uint64_t)(((kk >> 2) * TC_OWN_ROWS * 128 + (kk & 3) * 32) >> 4);
+        const uint64_t off_b = (uint64_t)(((kk >> 2) * ROWS_B * 128 + (kk & 3) * 32) >> 4);
+        ptx::mma_ss(d, a + off_a, b + off_b, idesc, (accumulate || kk > 0) ? 1u : 0u);
+    }
+}
+
+// Score MMAs of one tile:  S = X0 Y0^T,  Sd = X1 Y0^T + X0 Y1^T  per score pair.
+template <int KS, int NPAIR, int BC>
+__device__ __forceinline__ void issue_score_mmas(const uint64_t* xd, const uint64_t* yd, uint32_t dbase, uint32_t idesc) {
+#pragma unroll
+    for (int pr = 0; pr < NPAIR; ++pr) {
+        const uint32_t dS = dbase + 2 * pr * BC, dT = dS + BC;
+        issue_kmajor_gemm<KS, BC>(dS, xd[2 * pr], yd[2 * pr], idesc, false);
+        issue_kmajor_gemm<KS, BC>(dT, xd[2 * pr + 1], yd[2 * pr], idesc, false);
+        issue_kmajor_gemm<KS, BC>(dT, xd[2 * pr], yd[2 * pr + 1], idesc, true);
+    }
+}
+
+template <int NPAIR, int BC>
+__device__ __forceinline__ void issue_score_mmas_dyn(int ksteps, const uint64_t* xd, const uint64_t* yd, uint32_t dbase,
+                                                     uint32_t idesc) {
+    switch (ksteps) {
+        case 1: issue_score_mmas<1, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        case 2: issue_score_mmas<2, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        case 3: issue_score_mmas<3, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        case 4: issue_score_mmas<4, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        case 5: issue_score_mmas<5, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        case 6: issue_score_mmas<6, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        case 7: issue_score_mmas<7, NPAIR, BC>(xd, yd, dbase, idesc); break;
+        default: issue_score_mmas<8, NPAIR, BC>(xd, yd, dbase, idesc); break;
+    }
+}
+
+// Output MMAs of one tile:  acc0 += A0 B0,  acc1 += A1 B0 + A0 B1  with A from TMEM (operand of
+// k-step u at column 16u of its score accumulator) and B MN-major (k-step u = 16 stream rows = 2048 B).
+template <int BC>
+__device__ __forceinline__ void issue_output_mmas(uint32_t acc0, uint32_t acc1, uint32_t a0, uint32_t a1, uint64_t b0,
+                                                  uint64_t b1, uint32_t idesc, bool accumulate) {
+#pragma unroll
+    for (int u = 0; u < BC / 16; ++u) {
+        const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+        const uint32_t acc = (accumulate || u > 0) ? 1u : 0u;
+        ptx::mma_ts(acc0, a0 + 16 * u, b0 + off, idesc, acc);
+        ptx::mma_ts(acc1, a1 + 16 * u, b0 + off, idesc, acc);
+        ptx::mma_ts(acc1, a0 + 16 * u, b1 + off, idesc, 1u);
+    }
+}
 
 template <int MODE, int NA>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -118,7 +177,7 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 8 * 64);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 8 * 64 + 16);
     float* stats = reinterpret_cast<float*>(misc + 8 * 64 + 64);  // [stage][4][64]
-    float* xchg = stats + TC_STATS_STAGES * 4 * 64;               // [2][2][128]
+    float* xchg = stats + TC_STATS_STAGES * 4 * 64;               // [parity][half][value][128]
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -199,14 +258,11 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
         if (lane == 0) {
             const uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
             const uint32_t idesc_o = ptx::idesc_bf16_f32(128, p.dp, 0, 1);
-            // K-major descriptor of k-step kk (16 columns of d) of a tile with `rows` rows.
-            auto kdesc = [&](uint32_t tile, int rows, int kk) -> uint64_t {
-                return ptx::smem_desc_sw128(tile + (kk >> 2) * rows * 128 + (kk & 3) * 32, 16, 1024);
-            };
-            // MN-major descriptor (d is the MMA N dim) of k-step u (16 stream rows) of a stream tile.
-            auto ndesc = [&](uint32_t tile, int u) -> uint64_t {
-                return ptx::smem_desc_sw128(tile + u * 16 * 128, BC * 128, 1024);
-            };
+            // descriptors of the resident owner tiles (K-major) never change
+            uint64_t xd[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                xd[t] = ptx::smem_desc_sw128(own_base + (t < C::NOWN ? t : 0) * C::OWN_BYTES, 16, 1024);
             bool ok = ptx::mbar_wait(bar(C::B_OWNER), 0, abort_flag, TC_WAIT_LIMIT_NS);
             auto issue_scores = [&](int j) -> bool {
                 const int b = j & 1;
@@ -214,18 +270,10 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 if (NPAIR == 2)
                     if (!ptx::mbar_wait(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
                 ptx::tc_fence_after_sync();
-                for (int pr = 0; pr < NPAIR; ++pr) {
-                    const uint32_t x0 = own_base + (2 * pr) * C::OWN_BYTES, x1 = x0 + C::OWN_BYTES;
-                    const uint32_t y0 = stream_addr(2 * pr, j), y1 = stream_addr(2 * pr + 1, j);
-                    const uint32_t dS = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS + (2 * pr) * BC;
-                    const uint32_t dT = dS + BC;
-                    for (int kk = 0; kk < ksteps; ++kk)
-                        ptx::mma_ss(dS, kdesc(x0, TC_OWN_ROWS, kk), kdesc(y0, BC, kk), idesc_s, kk > 0);
-                    for (int kk = 0; kk < ksteps; ++kk)
-                        ptx::mma_ss(dT, kdesc(x1, TC_OWN_ROWS, kk), kdesc(y0, BC, kk), idesc_s, kk > 0);
-                    for (int kk = 0; kk < ksteps; ++kk)
-                        ptx::mma_ss(dT, kdesc(x0, TC_OWN_ROWS, kk), kdesc(y1, BC, kk), idesc_s, 1);
-                }
+                uint64_t yd[4];
+#pragma unroll
+                for (int t = 0; t < 2 * NPAIR; ++t) yd[t] = ptx::smem_desc_sw128(stream_addr(t, j), 16, 1024);
+                issue_score_mmas_dyn<NPAIR, BC>(ksteps, xd, yd, tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, idesc_s);
                 ptx::mma_commit(bar(C::B_SFULL + b));
                 ptx::mma_commit(bar(C::B_EEMPTY + j % SE));
                 return true;
@@ -237,14 +285,10 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 if (!ptx::mbar_wait(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
                 ptx::tc_fence_after_sync();
                 const uint32_t a0 = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
-                const uint32_t b0 = stream_addr(L_FIRST, j), b1 = stream_addr(L_FIRST + 1, j);
-                const uint32_t acc0 = tmem_base + C::COL_ACC0, acc1 = tmem_base + C::COL_ACC1;
-                for (int u = 0; u < BC / 16; ++u) {
-                    const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                    ptx::mma_ts(acc0, a0 + 16 * u, ndesc(b0, u), idesc_o, acc);
-                    ptx::mma_ts(acc1, a1 + 16 * u, ndesc(b0, u), idesc_o, acc);
-                    ptx::mma_ts(acc1, a0 + 16 * u, ndesc(b1, u), idesc_o, 1u);
-                }
+                // MN-major: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
+                const uint64_t b0 = ptx::smem_desc_sw128(stream_addr(L_FIRST, j), BC * 128, 1024);
+                const uint64_t b1 = ptx::smem_desc_sw128(stream_addr(L_FIRST + 1, j), BC * 128, 1024);
+                issue_output_mmas<BC>(tmem_base + C::COL_ACC0, tmem_base + C::COL_ACC1, a0, a1, b0, b1, idesc_o, j > 0);
                 ptx::mma_commit(bar(C::B_LEMPTY + j % SL));
                 ptx::mma_commit(bar(C::B_OUTDONE));
                 if (j == T - 1) ptx::mma_commit(bar(C::B_FINAL));
@@ -287,7 +331,14 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
         bool ok = true;
 
         if (MODE == MODE_FWD) {
-            float m_ref = -CUDART_INF_F, l = 0.f, mt = 0.f;
+            // Online softmax with two refinements.  (1) The reference maximum m_ref follows the true
+            // running maximum lazily: accumulators are rescaled only when a tile maximum exceeds it by
+            // more than TC_RESCALE_THRESHOLD (log2 units).  (2) The tangent weights are centred,
+            // T - c, with c the value of T at the row's running arg-max key, so that the bf16 rounding
+            // of P~*(T - c) is small where P~ is large; tO = R'/l - (mu - c) O with R' = sum P~ (T - c) V.
+            // c moves only when a new row maximum arrives whose T differs from c by more than
+            // TC_CENTER_DELTA; then R' += (c_old - c_new) O~ keeps the accumulators consistent.
+            float m_ref = -CUDART_INF_F, m_true = -CUDART_INF_F, cen = 0.f, l = 0.f, mt = 0.f;
             const int col0 = g * 32;
             for (int j = 0; j < T; ++j) {
                 const int b = j & 1;
@@ -309,42 +360,75 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 }
 #endif
                 const int nvalid = p.N - j * BC - col0;  // columns of this half that are real keys
-                float mx = -CUDART_INF_F;
-                if (nvalid >= 32) {
+                if (nvalid < 32) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
+                    for (int c = 0; c < 32; ++c)
                         if (c >= nvalid) s[c] = __float_as_uint(-CUDART_INF_F);
-                        mx = fmaxf(mx, __uint_as_float(s[c]));
+                }
+                // maximum of this half and the tangent score at that key (pairwise tree: short dependency chain)
+                float mx, tw;
+                {
+                    float vm[16], vt[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float a = __uint_as_float(s[2 * c]), b2 = __uint_as_float(s[2 * c + 1]);
+                        const bool gt = b2 > a;
+                        vm[c] = gt ? b2 : a;
+                        vt[c] = gt ? __uint_as_float(ts[2 * c + 1]) : __uint_as_float(ts[2 * c]);
                     }
+#pragma unroll
+                    for (int w = 8; w >= 1; w >>= 1) {
+#pragma unroll
+                        for (int c = 0; c < w; ++c) {
+                            const bool gt = vm[c + w] > vm[c];
+                            vm[c] = gt ? vm[c + w] : vm[c];
+                            vt[c] = gt ? vt[c + w] : vt[c];
+                        }
+                    }
+                    mx = vm[0];
+                    tw = vt[0];
                 }
                 mx *= p.c2;
+                tw *= p.alpha;
                 // the two threads that share a row (one per warpgroup) agree on the tile maximum
-                xchg[((j & 1) * 2 + g) * 128 + row] = mx;
+                float* xslot = xchg + (j & 1) * 512;
+                xslot[g * 256 + row] = mx;
+                xslot[g * 256 + 128 + row] = tw;
                 ptx::mbar_arrive(bar(C::B_XCHG + q));
                 if (!ptx::mbar_wait(bar(C::B_XCHG + q), j & 1, abort_flag, TC_WAIT_LIMIT_NS)) { ok = false; break; }
-                mx = fmaxf(mx, xchg[((j & 1) * 2 + (g ^ 1)) * 128 + row]);
-                const float m_new = fmaxf(m_ref, mx);
-                const bool need = m_new > m_ref + TC_RESCALE_THRESHOLD;
-                if (__any_sync(0xffffffffu, need)) {
-                    const float scale = need ? ptx::ex2(m_ref - m_new) : 1.0f;
-                    if (need) m_ref = m_new;
+                {
+                    const float omx = xslot[(g ^ 1) * 256 + row], otw = xslot[(g ^ 1) * 256 + 128 + row];
+                    const bool other_wins = (g == 0) ? (omx > mx) : (omx >= mx);  // ties go to half 0
+                    tw = other_wins ? otw : tw;
+                    mx = fmaxf(mx, omx);
+                }
+                const bool need_scale = mx > m_ref + TC_RESCALE_THRESHOLD;
+                const bool need_cen = (mx > m_true) && (j == 0 || fabsf(tw - cen) > TC_CENTER_DELTA);
+                m_true = fmaxf(m_true, mx);
+                if (__any_sync(0xffffffffu, need_scale || need_cen)) {
+                    const float scale = need_scale ? ptx::ex2(m_ref - mx) : 1.0f;
+                    const float fix = need_cen ? cen - tw : 0.f;
+                    if (need_scale) m_ref = mx;
+                    if (need_cen) cen = tw;
+                    mt = scale * fmaf(fix, l, mt);
                     l *= scale;
-                    mt *= scale;
                     if (j > 0) {
                         // accumulators must be at rest: the output MMAs of tile j-1 have completed
                         if (!ptx::mbar_wait(bar(C::B_OUTDONE), (j - 1) & 1, abort_flag, TC_WAIT_LIMIT_NS)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
-                        const uint32_t acc = lane_addr + (g == 0 ? C::COL_ACC0 : C::COL_ACC1);
-                        for (int ch = 0; ch < ksteps; ++ch) {
-                            uint32_t r[16];
-                            ptx::tmem_ld16(acc + 16 * ch, r);
+                        for (int ch = g; ch < ksteps; ch += 2) {
+                            uint32_t o[16], r[16];
+                            ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
+                            ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, r);
                             ptx::tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 16; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * scale);
-                            ptx::tmem_st16(acc + 16 * ch, r);
+                            for (int c = 0; c < 16; ++c) {
+                                const float ov = __uint_as_float(o[c]);
+                                r[c] = __float_as_uint(scale * fmaf(fix, ov, __uint_as_float(r[c])));
+                                o[c] = __float_as_uint(scale * ov);
+                            }
+                            ptx::tmem_st16(lane_addr + C::COL_ACC0 + 16 * ch, o);
+                            ptx::tmem_st16(lane_addr + C::COL_ACC1 + 16 * ch, r);
                         }
                     }
                 }
@@ -353,8 +437,8 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 for (int c = 0; c < 32; c += 2) {
                     const float p0 = ptx::ex2(fmaf(__uint_as_float(s[c]), p.c2, -m_ref));
                     const float p1 = ptx::ex2(fmaf(__uint_as_float(s[c + 1]), p.c2, -m_ref));
-                    const float t0 = p0 * (p.alpha * __uint_as_float(ts[c]));
-                    const float t1 = p1 * (p.alpha * __uint_as_float(ts[c + 1]));
+                    const float t0 = p0 * fmaf(p.alpha, __uint_as_float(ts[c]), -cen);
+                    const float t1 = p1 * fmaf(p.alpha, __uint_as_float(ts[c + 1]), -cen);
                     l += p0 + p1;
                     mt += t0 + t1;
                     pp[c >> 1] = ptx::pack_bf16(p0, p1);
@@ -369,18 +453,20 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar(C::B_PREADY + b));
             }
-            // ---- epilogue: O = O~/l, mu = mu~/l, tO = R/l - mu O, lse = ln2 (m + log2 l)
+            // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R'/l - (mu - c) O, lse = ln2 (m_ref + log2 l)
             if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, TC_WAIT_LIMIT_NS);
             if (ok) {
                 ptx::tc_fence_after_sync();
-                xchg[(0 * 2 + g) * 128 + row] = l;
-                xchg[(1 * 2 + g) * 128 + row] = mt;
+                float* xslot = xchg + (T & 1) * 512;
+                xslot[g * 256 + row] = l;
+                xslot[g * 256 + 128 + row] = mt;
                 ptx::mbar_arrive(bar(C::B_XCHG + q));
                 ok = ptx::mbar_wait(bar(C::B_XCHG + q), T & 1, abort_flag, TC_WAIT_LIMIT_NS);
             }
             if (ok) {
-                l += xchg[(0 * 2 + (g ^ 1)) * 128 + row];
-                mt += xchg[(1 * 2 + (g ^ 1)) * 128 + row];
+                const float* xslot = xchg + (T & 1) * 512;
+                l += xslot[(g ^ 1) * 256 + row];
+                mt += xslot[(g ^ 1) * 256 + 128 + row];
                 const float inv = 1.0f / l;
                 const float mun = mt * inv;
                 __nv_bfloat16* o_ptr = reinterpret_cast<__nv_bfloat16*>(p.out0) + ((size_t)bh * p.N + row0 + row) * p.d;
@@ -410,7 +496,7 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 }
                 if (g == 0 && row_valid) {
                     p.lse_out[(size_t)bh * p.N + row0 + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
-                    p.mu_out[(size_t)bh * p.N + row0 + row] = mun;
+                    p.mu_out[(size_t)bh * p.N + row0 + row] = cen + mun;
                 }
             }
         } else {

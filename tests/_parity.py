@@ -11,11 +11,14 @@ BWD_NAMES = ("dQ", "dK", "dV", "dtQ", "dtK", "dtV")
 
 
 def rel_err(got, ref):
+    """max|got - ref| / max|ref|.  A reference that is identically zero (e.g. dQ when N = 1) has no
+    scale of its own; its error is then reported in absolute terms (inputs are O(1))."""
     ref = np.asarray(ref, dtype=np.float64)
     got = np.asarray(got, dtype=np.float64)
     if not np.all(np.isfinite(got)):
         return float("inf")
-    return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-300))
+    scale = float(np.abs(ref).max())
+    return float(np.abs(got - ref).max() / (scale if scale > 1e-12 else 1.0))
 
 
 def run_case(wl, oracle_heads=None, dtype=torch.bfloat16, flags=0, scale=0.0, device="cuda:0"):
