@@ -110,7 +110,7 @@ __device__ __forceinline__ void issue_kmajor_gemm(uint32_t d, uint64_t a, uint64
     for (int kk = 0; kk < KS; ++kk) {
         const uint64_t off_a = (uint64_t)(((kk >> 2) * TC_OWN_ROWS * 128 + (kk & 3) * 32) >> 4);
         const uint64_t off_b = (uint64_t)(((kk >> 2) * ROWS_B * 128 + (kk & 3) * 32) >> 4);
-        ptx::mma_ss(d, a + off_a, b + off_b, idesc, (accumulate || kk > 0) ? 1u : 0u);
+        ptx::mma_ss_elect(d, a + off_a, b + off_b, idesc, (accumulate || kk > 0) ? 1u : 0u);
     }
 }
 
@@ -150,9 +150,9 @@ __device__ __forceinline__ void issue_output_mmas(uint32_t acc0, uint32_t acc1, 
     for (int u = 0; u < BC / 16; ++u) {
         const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
         const uint32_t acc = (accumulate || u > 0) ? 1u : 0u;
-        ptx::mma_ts(acc0, a0 + 16 * u, b0 + off, idesc, acc);
-        ptx::mma_ts(acc1, a1 + 16 * u, b0 + off, idesc, acc);
-        ptx::mma_ts(acc1, a0 + 16 * u, b1 + off, idesc, 1u);
+        ptx::mma_ts_elect(acc0, a0 + 16 * u, b0 + off, idesc, acc);
+        ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc, acc);
+        ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc, 1u);
     }
 }
 
@@ -255,7 +255,7 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        {   // the whole warp runs the loop; one elected lane issues (see mma_ts_elect)
             const uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
             const uint32_t idesc_o = ptx::idesc_bf16_f32(128, p.dp, 0, 1);
             // descriptors of the resident owner tiles (K-major) never change
@@ -263,35 +263,35 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
 #pragma unroll
             for (int t = 0; t < 4; ++t)
                 xd[t] = ptx::smem_desc_sw128(own_base + (t < C::NOWN ? t : 0) * C::OWN_BYTES, 16, 1024);
-            bool ok = ptx::mbar_wait(bar(C::B_OWNER), 0, abort_flag, TC_WAIT_LIMIT_NS);
+            bool ok = ptx::mbar_wait_warp(bar(C::B_OWNER), 0, abort_flag, TC_WAIT_LIMIT_NS);
             auto issue_scores = [&](int j) -> bool {
                 const int b = j & 1;
-                if (!ptx::mbar_wait(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
+                if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
                 if (NPAIR == 2)
-                    if (!ptx::mbar_wait(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
+                    if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
                 ptx::tc_fence_after_sync();
                 uint64_t yd[4];
 #pragma unroll
                 for (int t = 0; t < 2 * NPAIR; ++t) yd[t] = ptx::smem_desc_sw128(stream_addr(t, j), 16, 1024);
                 issue_score_mmas_dyn<NPAIR, BC>(ksteps, xd, yd, tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, idesc_s);
-                ptx::mma_commit(bar(C::B_SFULL + b));
-                ptx::mma_commit(bar(C::B_EEMPTY + j % SE));
+                ptx::mma_commit_elect(bar(C::B_SFULL + b));
+                ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
                 return true;
             };
             auto issue_outputs = [&](int j) -> bool {
                 const int b = j & 1;
                 if (NPAIR == 1)
-                    if (!ptx::mbar_wait(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
-                if (!ptx::mbar_wait(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
+                    if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
+                if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, TC_WAIT_LIMIT_NS)) return false;
                 ptx::tc_fence_after_sync();
                 const uint32_t a0 = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
                 // MN-major: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
                 const uint64_t b0 = ptx::smem_desc_sw128(stream_addr(L_FIRST, j), BC * 128, 1024);
                 const uint64_t b1 = ptx::smem_desc_sw128(stream_addr(L_FIRST + 1, j), BC * 128, 1024);
                 issue_output_mmas<BC>(tmem_base + C::COL_ACC0, tmem_base + C::COL_ACC1, a0, a1, b0, b1, idesc_o, j > 0);
-                ptx::mma_commit(bar(C::B_LEMPTY + j % SL));
-                ptx::mma_commit(bar(C::B_OUTDONE));
-                if (j == T - 1) ptx::mma_commit(bar(C::B_FINAL));
+                ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+                ptx::mma_commit_elect(bar(C::B_OUTDONE));
+                if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
                 return true;
             };
             if (ok) ok = issue_scores(0);

@@ -1,0 +1,451 @@
+// Forward kernel of attention with a Jacobian-vector product on sm_100a (tcgen05 + TMEM + TMA),
+// for padded head dims up to 80 (d = 72 runs as 80).
+//
+// Per head (App. C Eq. "sdpa" and the definitions under "Step 1"):
+//     S = Q K^T, Sd = tQ K^T + Q tK^T            (three GEMMs per key tile, fp32 accumulators in TMEM)
+//     P~ = 2^(c2 S - m), T = alpha Sd             (element-wise warps; m is a lazily updated row reference)
+//     O~ += P~ V,  R += (P~ (T - c)) V + P~ tV    (three GEMMs per key tile)
+//     O = O~/l,  tO = R/l - (mu - c) O,  lse = ln2 (m + log2 l),  mu = c + sum(P~ (T - c))/l
+//
+// A CTA owns 128 query rows of one head and streams the keys in tiles of 64.
+//
+// What is where
+//   * Q and tQ of the CTA's rows are written once into tensor memory as bf16 operands, so the three
+//     score GEMMs read only their B operand (the K / tK tile) from shared memory.  With A taken from
+//     shared memory a 128 x 64 x 16 MMA would move 6 KB per 32 tensor-pipe cycles, more than the
+//     128 B/clk a shared-memory port delivers.
+//   * The score accumulators are double-buffered (2 x (64 + 64) columns); the bf16 operands P~ and
+//     P~(T - c) are written back over the columns of the accumulators they came from.
+//   * 16 element-wise warps: warp w works on TMEM lane quadrant w % 4 (32 query rows) and on the
+//     16-column slice w / 4 of every key tile, which is exactly one k-step of the value GEMMs.
+//
+// Online softmax without a per-tile dependency: the reference m of a row follows the running row
+// maximum lazily.  The four warps that share a row exchange their slice maxima through shared memory;
+// only when the tile maximum exceeds m by more than FWD_LAZY_LOG2 (rare after the first tile) do they
+// take the slow path together: m moves to the new maximum, the centre c of the tangent weights moves
+// to T at the new arg-max key, and the accumulators are rescaled, R += (c_old - c_new) O~ keeping them
+// consistent.  Centring T keeps the bf16 rounding of P~ (T - c) small where P~ is large, so that
+// tO = R/l - (mu - c) O does not cancel badly on rows with a peaked softmax.
+//
+// Every wait on an mbarrier is bounded; when one gives up the block records a time-out status and
+// all roles leave their loops.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "sm100_ptx.cuh"
+
+namespace tvm_attn {
+
+constexpr int FWD_THREADS = 640;        // 4 control warps + 16 element-wise warps
+constexpr int FWD_ROWS = 128;           // query rows per CTA
+constexpr int FWD_BC = 64;              // keys per tile
+constexpr float FWD_LAZY_LOG2 = 3.0f;   // slack of the row reference, in log2 units
+constexpr uint64_t FWD_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;
+
+struct FwdParams {
+    int N, d, BH;
+    float alpha;  // softmax scale
+    float c2;     // alpha * log2(e)
+    const __nv_bfloat16* Q;
+    const __nv_bfloat16* tQ;
+    __nv_bfloat16* O;
+    __nv_bfloat16* tO;
+    float* lse;
+    float* mu;
+    int* status;  // device status word; non-zero makes the kernel a no-op
+};
+
+template <int DP>
+struct FwdCfg {
+    static_assert(DP % 16 == 0 && DP >= 16 && DP <= 80, "padded head dim must be 16..80");
+    static constexpr int KS = DP / 16;            // k-steps of a score GEMM
+    static constexpr int NA = DP > 64 ? 2 : 1;    // 64-column swizzle atoms per row
+    static constexpr int ST_BYTES = NA * FWD_BC * 128;
+    static constexpr int SE = NA == 1 ? 4 : 3;    // stages of the (K, tK) ring
+    static constexpr int SL = NA == 1 ? 4 : 3;    // stages of the (V, tV) ring
+    static constexpr int TILE_BYTES = (SE + SL) * 2 * ST_BYTES;
+    // barrier slots
+    static constexpr int B_EFULL = 0;
+    static constexpr int B_EEMPTY = B_EFULL + SE;
+    static constexpr int B_LFULL = B_EEMPTY + SE;
+    static constexpr int B_LEMPTY = B_LFULL + SL;
+    static constexpr int B_SFULL = B_LEMPTY + SL;
+    static constexpr int B_PREADY = B_SFULL + 2;
+    static constexpr int B_OUTDONE = B_PREADY + 2;
+    static constexpr int B_FINAL = B_OUTDONE + 1;
+    static constexpr int B_QREADY = B_FINAL + 1;
+    static constexpr int B_XMAX = B_QREADY + 1;   // per quadrant: slice maxima exchanged
+    static constexpr int B_XSLOW = B_XMAX + 4;    // per quadrant: slow-path / epilogue exchange
+    static constexpr int NBARS = B_XSLOW + 4;
+    static_assert(NBARS <= 48, "barrier table too small");
+    static constexpr int XMAX_FLOATS = 2 * 128 * 4;   // [parity][row][slice]
+    static constexpr int XSLOW_FLOATS = 128 * 4 * 2;  // [row][slice][2]
+    static constexpr int MISC_BYTES = 48 * 8 + 64 + (XMAX_FLOATS + XSLOW_FLOATS) * 4;
+    static constexpr int SMEM_BYTES = TILE_BYTES + MISC_BYTES + 1024 /*alignment slack*/;
+    // TMEM columns: accumulators O~ and R, the bf16 operands Q and tQ in the gaps behind them, and
+    // two score buffers of (S | Sd).
+    static constexpr int COL_ACC0 = 0, COL_Q = DP, COL_ACC1 = 128, COL_TQ = 128 + DP, COL_SCORE = 256;
+    static constexpr int SCORE_BUF_COLS = 2 * FWD_BC;
+    static_assert(DP + DP / 2 <= 128, "operand does not fit behind its accumulator");
+};
+
+// Element-wise warps of the forward: `w` in 0..15, TMEM lane quadrant w & 3, column slice w >> 2.
+template <int DP>
+__device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tmem_base, uint32_t bar0,
+                                                volatile int* abort_flag, float* xmax, float* xslow, int w, int lane,
+                                                int bh, int row0, int T) {
+    using C = FwdCfg<DP>;
+    constexpr int BC = FWD_BC, KS = C::KS;
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
+    const int q = w & 3, sl = w >> 2;
+    const int row = q * 32 + lane;  // query row inside the CTA tile
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    const bool row_valid = row0 + row < p.N;
+    const size_t grow = (size_t)bh * p.N + row0 + row;
+
+    // ---- Q and tQ rows -> bf16 operands in tensor memory (k-step kk at 8 packed columns)
+    for (int ch = sl; ch < 2 * KS; ch += 4) {
+        const bool is_t = ch >= KS;
+        const int kk = is_t ? ch - KS : ch;
+        const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow * p.d + 16 * kk;
+        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+        if (row_valid && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
+        if (row_valid && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
+        const uint32_t r[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        ptx::tmem_st8(lane_addr + (is_t ? C::COL_TQ : C::COL_Q) + 8 * kk, r);
+    }
+    ptx::tmem_wait_st();
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+
+    float m_ref = -CUDART_INF_F, cen = 0.f;
+    uint64_t l2 = 0ull, mt2 = 0ull;  // two partial sums each of P~ and of P~(T - c) over this warp's slices
+    int n_slow = 0;                  // exchanges done on B_XSLOW
+    bool ok = true;
+    const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
+    float2* xs2 = reinterpret_cast<float2*>(xslow);
+
+    for (int j = 0; j < T; ++j) {
+        const int b = j & 1;
+        if (!ptx::mbar_wait(bar(C::B_SFULL + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS;
+        uint32_t s[16], ts[16];
+        ptx::tmem_ld16(sbase + 16 * sl, s);
+        ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
+        ptx::tmem_wait_ld();
+        const int nvalid = p.N - j * BC - 16 * sl;  // columns of this slice that are real keys
+        if (nvalid < 16) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+                if (c >= nvalid) s[c] = __float_as_uint(-CUDART_INF_F);
+        }
+        // slice maximum, exchanged with the three other warps of this quadrant
+        float mx = ptx::max3(__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(s[2]));
+#pragma unroll
+        for (int c = 3; c < 15; c += 2) mx = ptx::max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+        mx = fmaxf(mx, __uint_as_float(s[15]));
+        float* xm = xmax + (j & 1) * 512;
+        xm[row * 4 + sl] = mx;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_XMAX + q));
+        if (!ptx::mbar_wait(bar(C::B_XMAX + q), j & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        const float4 o4 = *reinterpret_cast<const float4*>(xm + row * 4);
+        const float mrow = fmaxf(ptx::max3(o4.x, o4.y, o4.z), o4.w) * p.c2;  // tile maximum of the row, log2 units
+        const bool need = mrow > m_ref + FWD_LAZY_LOG2;
+        if (__any_sync(0xffffffffu, need)) {
+            // ---- slow path, taken by the four warps of the quadrant together
+            float la = -CUDART_INF_F, lt = 0.f;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const bool gt = __uint_as_float(s[c]) > la;
+                la = gt ? __uint_as_float(s[c]) : la;
+                lt = gt ? __uint_as_float(ts[c]) : lt;
+            }
+            xs2[row * 4 + sl] = make_float2(la, lt);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
+            if (!ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            ++n_slow;
+            float ba = -CUDART_INF_F, bt = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {  // ties go to the lowest slice
+                const float2 v = xs2[row * 4 + k];
+                const bool gt = v.x > ba;
+                ba = gt ? v.x : ba;
+                bt = gt ? v.y : bt;
+            }
+            const float tw = bt * p.alpha;
+            const float scale = need ? ptx::ex2(m_ref - mrow) : 1.0f;
+            const float fix = need ? cen - tw : 0.f;
+            if (need) { m_ref = mrow; cen = tw; }
+            {
+                float l0, l1, t0, t1;
+                ptx::unpack2(l2, l0, l1);
+                ptx::unpack2(mt2, t0, t1);
+                t0 = scale * fmaf(fix, l0, t0);
+                t1 = scale * fmaf(fix, l1, t1);
+                l0 *= scale;
+                l1 *= scale;
+                l2 = ptx::pack2(l0, l1);
+                mt2 = ptx::pack2(t0, t1);
+            }
+            if (j > 0) {
+                // accumulators must be at rest: the value MMAs of tile j-1 have completed
+                if (!ptx::mbar_wait(bar(C::B_OUTDONE), (j - 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                for (int ch = sl; ch < KS; ch += 4) {
+                    uint32_t o[16], r[16];
+                    ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
+                    ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, r);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float ov = __uint_as_float(o[c]);
+                        r[c] = __float_as_uint(scale * fmaf(fix, ov, __uint_as_float(r[c])));
+                        o[c] = __float_as_uint(scale * ov);
+                    }
+                    ptx::tmem_st16(lane_addr + C::COL_ACC0 + 16 * ch, o);
+                    ptx::tmem_st16(lane_addr + C::COL_ACC1 + 16 * ch, r);
+                }
+            }
+        }
+        // ---- P~ = 2^(c2 s - m), P~ (T - c); two elements per instruction where the hardware allows
+        const uint64_t nm = ptx::pack2(-m_ref, -m_ref), nc = ptx::pack2(-cen, -cen);
+        uint32_t pp[8], ppt[8];
+#pragma unroll
+        for (int c = 0; c < 16; c += 2) {
+            const uint64_t x2 = ptx::fma2(ptx::pack2u(s[c], s[c + 1]), c2c2, nm);
+            float x0, x1;
+            ptx::unpack2(x2, x0, x1);
+            const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+            const uint64_t p2 = ptx::pack2(p0, p1);
+            const uint64_t t2 = ptx::fma2(ptx::pack2u(ts[c], ts[c + 1]), aa, nc);
+            const uint64_t pt2 = ptx::mul2(p2, t2);
+            l2 = ptx::add2(l2, p2);
+            mt2 = ptx::add2(mt2, pt2);
+            float q0, q1;
+            ptx::unpack2(pt2, q0, q1);
+            pp[c >> 1] = ptx::pack_bf16(p0, p1);
+            ppt[c >> 1] = ptx::pack_bf16(q0, q1);
+        }
+        // operand of k-step `sl` (16 keys) sits at column 16*sl of the accumulator it replaces
+        ptx::tmem_st8(sbase + 16 * sl, pp);
+        ptx::tmem_st8(sbase + BC + 16 * sl, ppt);
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
+    }
+
+    // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R/l - (mu - c) O, lse = ln2 (m + log2 l)
+    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, FWD_WAIT_LIMIT_NS);
+    if (ok) {
+        ptx::tc_fence_after_sync();
+        float l0, l1, t0, t1;
+        ptx::unpack2(l2, l0, l1);
+        ptx::unpack2(mt2, t0, t1);
+        xs2[row * 4 + sl] = make_float2(l0 + l1, t0 + t1);
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
+        ok = ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+    }
+    if (ok) {
+        float l = 0.f, mt = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float2 v = xs2[row * 4 + k];
+            l += v.x;
+            mt += v.y;
+        }
+        const float inv = 1.0f / l;
+        const float mun = mt * inv;
+        __nv_bfloat16* o_ptr = p.O + grow * p.d;
+        __nv_bfloat16* t_ptr = p.tO + grow * p.d;
+        for (int ch = sl; ch < KS; ch += 4) {
+            uint32_t o[16], r[16];
+            ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
+            ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, r);
+            ptx::tmem_wait_ld();
+            uint32_t po[8], pt[8];
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) {
+                const float o0 = __uint_as_float(o[c]) * inv, o1 = __uint_as_float(o[c + 1]) * inv;
+                const float r0 = fmaf(-mun, o0, __uint_as_float(r[c]) * inv);
+                const float r1 = fmaf(-mun, o1, __uint_as_float(r[c + 1]) * inv);
+                po[c >> 1] = ptx::pack_bf16(o0, o1);
+                pt[c >> 1] = ptx::pack_bf16(r0, r1);
+            }
+            if (row_valid) {
+                *reinterpret_cast<uint4*>(o_ptr + 16 * ch) = make_uint4(po[0], po[1], po[2], po[3]);
+                *reinterpret_cast<uint4*>(t_ptr + 16 * ch) = make_uint4(pt[0], pt[1], pt[2], pt[3]);
+                if (16 * ch + 8 < p.d) {
+                    *reinterpret_cast<uint4*>(o_ptr + 16 * ch + 8) = make_uint4(po[4], po[5], po[6], po[7]);
+                    *reinterpret_cast<uint4*>(t_ptr + 16 * ch + 8) = make_uint4(pt[4], pt[5], pt[6], pt[7]);
+                }
+            }
+        }
+        if (sl == 0 && row_valid) {
+            p.lse[grow] = (m_ref + log2f(l)) * 0.6931471805599453f;
+            p.mu[grow] = cen + mun;
+        }
+    }
+}
+
+template <int DP>
+__global__ void __launch_bounds__(FWD_THREADS, 1)
+jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_tk,
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tv,
+               const FwdParams p) {
+    using C = FwdCfg<DP>;
+    constexpr int BC = FWD_BC, KS = C::KS, NA = C::NA, SE = C::SE, SL = C::SL;
+    if (*reinterpret_cast<volatile int*>(p.status) != 0) return;  // an earlier kernel timed out
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t e_base = ptx::smem_u32(smem);
+    const uint32_t l_base = e_base + SE * 2 * C::ST_BYTES;
+    uint8_t* misc = smem + C::TILE_BYTES;
+    const uint32_t bar0 = ptx::smem_u32(misc);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 48 * 8 + 16);
+    float* xmax = reinterpret_cast<float*>(misc + 48 * 8 + 64);
+    float* xslow = xmax + C::XMAX_FLOATS;
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row_tiles = (p.N + FWD_ROWS - 1) / FWD_ROWS;
+    const int bh = blockIdx.x / row_tiles;
+    const int row0 = (blockIdx.x - bh * row_tiles) * FWD_ROWS;
+    const int T = (p.N + BC - 1) / BC;  // key tiles
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), 1); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
+        for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), 1); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(bar(C::B_SFULL + b), 1);
+            ptx::mbar_init(bar(C::B_PREADY + b), 16);
+        }
+        ptx::mbar_init(bar(C::B_OUTDONE), 1);
+        ptx::mbar_init(bar(C::B_FINAL), 1);
+        ptx::mbar_init(bar(C::B_QREADY), 16);
+        for (int q = 0; q < 4; ++q) { ptx::mbar_init(bar(C::B_XMAX + q), 4); ptx::mbar_init(bar(C::B_XSLOW + q), 4); }
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // shared-memory address of tile `t` (0 = K, 1 = tK in the E ring; 2 = V, 3 = tV in the L ring) of iteration j
+    auto tile_addr = [&](int t, int j) -> uint32_t {
+        return t < 2 ? e_base + ((j % SE) * 2 + t) * C::ST_BYTES : l_base + ((j % SL) * 2 + (t - 2)) * C::ST_BYTES;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const CUtensorMap* maps[4] = {&tm_k, &tm_tk, &tm_v, &tm_tv};
+            for (int j = 0; j < T; ++j) {
+                for (int ring = 0; ring < 2; ++ring) {
+                    const int S = ring == 0 ? SE : SL;
+                    const int s = j % S, ph = (j / S) & 1;
+                    const int full = (ring == 0 ? C::B_EFULL : C::B_LFULL) + s;
+                    const int empty = (ring == 0 ? C::B_EEMPTY : C::B_LEMPTY) + s;
+                    if (!ptx::mbar_wait(bar(empty), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS)) goto producer_done;
+                    ptx::mbar_arrive_expect_tx(bar(full), 2 * C::ST_BYTES);
+                    for (int t = 2 * ring; t < 2 * ring + 2; ++t)
+                        for (int a = 0; a < NA; ++a)
+                            ptx::tma_load_3d(tile_addr(t, j) + a * BC * 128, maps[t], bar(full), a * 64, j * BC, bh);
+                }
+            }
+        producer_done:;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        {   // the whole warp runs the loop; one elected lane issues (see mma_ts_elect)
+            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
+            constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
+            const uint32_t aq = tmem_base + C::COL_Q, atq = tmem_base + C::COL_TQ;
+            auto issue_scores = [&](int j) -> bool {
+                const int b = j & 1;
+                if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
+                ptx::tc_fence_after_sync();
+                const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
+                const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
+                const uint32_t dS = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {  // S = Q K^T
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dS, aq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {  // Sd = tQ K^T
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dT, atq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {  // Sd += Q tK^T
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
+                }
+                ptx::mma_commit_elect(bar(C::B_SFULL + b));
+                ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+                return true;
+            };
+            auto issue_outputs = [&](int j) -> bool {
+                const int b = j & 1;
+                if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
+                if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
+                ptx::tc_fence_after_sync();
+                const uint32_t a0 = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
+                // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
+                const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
+                const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+                const uint32_t acc0 = tmem_base + C::COL_ACC0, acc1 = tmem_base + C::COL_ACC1;
+#pragma unroll
+                for (int u = 0; u < BC / 16; ++u) {
+                    const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                    const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                    ptx::mma_ts_elect(acc0, a0 + 16 * u, vd + off, idesc_o, acc);   // O~ += P~ V
+                    ptx::mma_ts_elect(acc1, a1 + 16 * u, vd + off, idesc_o, acc);   // R  += P~(T-c) V
+                    ptx::mma_ts_elect(acc1, a0 + 16 * u, tvd + off, idesc_o, 1u);   // R  += P~ tV
+                }
+                ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+                ptx::mma_commit_elect(bar(C::B_OUTDONE));
+                if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                return true;
+            };
+            bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, FWD_WAIT_LIMIT_NS);
+            ptx::tc_fence_after_sync();
+            if (ok) ok = issue_scores(0);
+            for (int j = 0; ok && j < T; ++j) {
+                if (j + 1 < T) ok = issue_scores(j + 1);
+                if (ok) ok = issue_outputs(j);
+            }
+        }
+    } else if (warp >= 4) {
+        fwd_elementwise<DP>(p, tmem_base, bar0, abort_flag, xmax, xslow, warp - 4, lane, bh, row0, T);
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, 1);
+}
+
+}  // namespace tvm_attn

@@ -12,6 +12,7 @@
 #include <mutex>
 
 #include "dual_attn_sm100.cuh"
+#include "jvp_fwd_sm100.cuh"
 #include "simt_kernels.cuh"
 
 namespace tvm_attn {
@@ -196,6 +197,26 @@ static int launch_tc_na(const Shape& s, const void* const own[4], const void* co
     return s.d <= 64 ? launch_tc<MODE, 1>(s, own, strm, prm, st) : launch_tc<MODE, 2>(s, own, strm, prm, st);
 }
 
+// Forward for padded head dims up to 80: operands Q, tQ live in tensor memory (jvp_fwd_sm100.cuh).
+template <int DP>
+static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams& prm, cudaStream_t st) {
+    using C = FwdCfg<DP>;
+    CUtensorMap m[4];
+    for (int t = 0; t < 4; ++t) {
+        const int rc = make_tmap(&m[t], strm[t], s, FWD_BC);
+        if (rc != TVM_ATTN_OK) return rc;
+    }
+    auto kern = jvp_fwd_kernel<DP>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        return TVM_ATTN_CUDA_ERROR;
+    const long long grid = s.BH * ((s.N + FWD_ROWS - 1) / FWD_ROWS);
+    g_prof.before(st);
+    kern<<<(unsigned)grid, FWD_THREADS, C::SMEM_BYTES, st>>>(m[0], m[1], m[2], m[3], prm);
+    g_prof.after(st);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
 #ifdef TVM_ATTN_DEBUG_DUMP
 static float* g_debug_dump = nullptr;
 #endif
@@ -247,10 +268,25 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
     if (rc != TVM_ATTN_OK) return rc;
     int* status = status_word_ptr();
     if (!status) return TVM_ATTN_CUDA_ERROR;
+    const void* strm[4] = {K, tK, V, tV};
+    if (s.dp <= 80) {
+        FwdParams f;
+        f.N = s.N; f.d = s.d; f.BH = (int)s.BH;
+        f.alpha = s.alpha; f.c2 = s.alpha * 1.4426950408889634f;
+        f.Q = static_cast<const __nv_bfloat16*>(Q); f.tQ = static_cast<const __nv_bfloat16*>(tQ);
+        f.O = static_cast<__nv_bfloat16*>(O); f.tO = static_cast<__nv_bfloat16*>(tO);
+        f.lse = lse; f.mu = mu; f.status = status;
+        switch (s.dp) {
+            case 16: return launch_fwd<16>(s, strm, f, st);
+            case 32: return launch_fwd<32>(s, strm, f, st);
+            case 48: return launch_fwd<48>(s, strm, f, st);
+            case 64: return launch_fwd<64>(s, strm, f, st);
+            default: return launch_fwd<80>(s, strm, f, st);
+        }
+    }
     TcParams prm = base_params(s, status);
     prm.out0 = O; prm.out1 = tO; prm.lse_out = lse; prm.mu_out = mu;
     const void* own[4] = {Q, tQ, Q, tQ};
-    const void* strm[4] = {K, tK, V, tV};
     return launch_tc_na<MODE_FWD>(s, own, strm, prm, st);
 }
 
