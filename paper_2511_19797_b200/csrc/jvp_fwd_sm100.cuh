@@ -52,11 +52,16 @@ struct FwdParams {
     float c2;     // alpha * log2(e)
     const __nv_bfloat16* Q;
     const __nv_bfloat16* tQ;
+    const __nv_bfloat16* K;   // the four streamed tensors, for the 16-byte copies of columns >= 64
+    const __nv_bfloat16* tK;
+    const __nv_bfloat16* V;
+    const __nv_bfloat16* tV;
     __nv_bfloat16* O;
     __nv_bfloat16* tO;
     float* lse;
     float* mu;
     int* status;  // device status word; non-zero makes the kernel a no-op
+    unsigned long long* tl;  // unused (timeline builds of other variants)
 };
 
 template <int DP>
@@ -68,6 +73,7 @@ struct FwdCfg {
     static constexpr int SE = NA == 1 ? 4 : 3;    // stages of the (K, tK) ring
     static constexpr int SL = NA == 1 ? 4 : 3;    // stages of the (V, tV) ring
     static constexpr int TILE_BYTES = (SE + SL) * 2 * ST_BYTES;
+    static constexpr int FULL_COUNT = NA;         // TMA issuer (+ the warp copying columns >= 64)
     // barrier slots
     static constexpr int B_EFULL = 0;
     static constexpr int B_EEMPTY = B_EFULL + SE;
@@ -326,8 +332,8 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), 1); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
-        for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), 1); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
+        for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
+        for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar(C::B_SFULL + b), 1);
             ptx::mbar_init(bar(C::B_PREADY + b), 16);
@@ -337,6 +343,19 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         ptx::mbar_init(bar(C::B_QREADY), 16);
         for (int q = 0; q < 4; ++q) { ptx::mbar_init(bar(C::B_XMAX + q), 4); ptx::mbar_init(bar(C::B_XSLOW + q), 4); }
         ptx::fence_mbar_init();
+    }
+    if (NA == 2) {
+        // Second swizzle atom of every stage: the 16-byte chunks behind the copied columns must read as
+        // zero (they pad d to a multiple of 16) and are never written again.  Logical chunk k of row r
+        // sits at physical chunk k ^ (r & 7).
+        if (((p.d - 64) >> 3) < 2) {
+            for (int i = threadIdx.x; i < (SE + SL) * 2 * BC; i += FWD_THREADS) {
+                const int tile = i / BC, r = i - tile * BC;
+                uint8_t* atom2 = smem + tile * C::ST_BYTES + BC * 128;
+                *reinterpret_cast<uint4*>(atom2 + r * 128 + ((1 ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            }
+            ptx::fence_proxy_async_smem();
+        }
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
@@ -352,25 +371,53 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         return t < 2 ? e_base + ((j % SE) * 2 + t) * C::ST_BYTES : l_base + ((j % SL) * 2 + (t - 2)) * C::ST_BYTES;
     };
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            const CUtensorMap* maps[4] = {&tm_k, &tm_tk, &tm_v, &tm_tv};
-            for (int j = 0; j < T; ++j) {
-                for (int ring = 0; ring < 2; ++ring) {
-                    const int S = ring == 0 ? SE : SL;
-                    const int s = j % S, ph = (j / S) & 1;
-                    const int full = (ring == 0 ? C::B_EFULL : C::B_LFULL) + s;
-                    const int empty = (ring == 0 ? C::B_EEMPTY : C::B_LEMPTY) + s;
-                    if (!ptx::mbar_wait(bar(empty), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS)) goto producer_done;
-                    ptx::mbar_arrive_expect_tx(bar(full), 2 * C::ST_BYTES);
-                    for (int t = 2 * ring; t < 2 * ring + 2; ++t)
-                        for (int a = 0; a < NA; ++a)
-                            ptx::tma_load_3d(tile_addr(t, j) + a * BC * 128, maps[t], bar(full), a * 64, j * BC, bh);
+    if (warp == 0 || warp == 2) {
+        // ------------------------------------------------------------------ producers: warp 0 feeds the
+        // (K, tK) ring, warp 2 the (V, tV) ring.  Lane 0 issues the TMA boxes of columns 0..63; all lanes
+        // copy the columns from 64 on, 16 bytes per row and chunk (a 64-column TMA box hanging over the
+        // end of a 144-byte row would read the next row's bytes from L2 only to replace them by zeros,
+        // which nearly doubled the L2 traffic), and signal them one tile later so that two tiles of copies
+        // are in flight.
+        const int ring = warp >> 1;
+        const int S = ring == 0 ? SE : SL;
+        const int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
+        const CUtensorMap* maps[2] = {ring == 0 ? &tm_k : &tm_v, ring == 0 ? &tm_tk : &tm_tv};
+        const __nv_bfloat16* srcs[2] = {ring == 0 ? p.K : p.V, ring == 0 ? p.tK : p.tV};
+        const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
+        bool ok = true;
+        for (int j = 0; j < T; ++j) {
+            const int s = j % S, ph = (j / S) & 1;
+            ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (!ok) break;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
+                for (int t = 0; t < 2; ++t) ptx::tma_load_3d(tile_addr(2 * ring + t, j), maps[t], bar(b_full + s), 0, j * BC, bh);
+            }
+            if constexpr (NA == 2) {
+                for (int i = lane; i < 2 * BC * ntail; i += 32) {
+                    const int t = i / (BC * ntail), rem = i - t * (BC * ntail);
+                    const int r = rem / ntail, k = rem - r * ntail;
+                    const int grow = j * BC + r;
+                    const bool v = grow < p.N;
+                    const __nv_bfloat16* src = srcs[t] + ((size_t)bh * p.N + (v ? grow : 0)) * p.d + 64 + 8 * k;
+                    ptx::cp_async_16(tile_addr(2 * ring + t, j) + BC * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+                }
+                ptx::cp_async_commit();
+                if (j > 0) {
+                    ptx::cp_async_wait<1>();
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(b_full + (j - 1) % S));
                 }
             }
-        producer_done:;
         }
+        if (NA == 2 && ok) {
+            ptx::cp_async_wait<0>();
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(b_full + (T - 1) % S));
+        }
+        if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         {   // the whole warp runs the loop; one elected lane issues (see mma_ts_elect)

@@ -220,6 +220,9 @@ static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams
 #ifdef TVM_ATTN_DEBUG_DUMP
 static float* g_debug_dump = nullptr;
 #endif
+#ifdef TVM_ATTN_TIMELINE
+static unsigned long long* g_timeline = nullptr;  // clock stamps of CTA 0 (timeline builds only)
+#endif
 
 static TcParams base_params(const Shape& s, int* status) {
     TcParams prm;
@@ -274,6 +277,13 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
         f.N = s.N; f.d = s.d; f.BH = (int)s.BH;
         f.alpha = s.alpha; f.c2 = s.alpha * 1.4426950408889634f;
         f.Q = static_cast<const __nv_bfloat16*>(Q); f.tQ = static_cast<const __nv_bfloat16*>(tQ);
+        f.K = static_cast<const __nv_bfloat16*>(K); f.tK = static_cast<const __nv_bfloat16*>(tK);
+        f.V = static_cast<const __nv_bfloat16*>(V); f.tV = static_cast<const __nv_bfloat16*>(tV);
+#ifdef TVM_ATTN_TIMELINE
+        f.tl = g_timeline;
+#else
+        f.tl = nullptr;
+#endif
         f.O = static_cast<__nv_bfloat16*>(O); f.tO = static_cast<__nv_bfloat16*>(tO);
         f.lse = lse; f.mu = mu; f.status = status;
         switch (s.dp) {
@@ -393,6 +403,9 @@ int tvm_attn_version(void) { return 100; }
 
 #ifdef TVM_ATTN_DEBUG_DUMP
 void tvm_attn_debug_set_dump(float* device_ptr) { g_debug_dump = device_ptr; }
+#endif
+#ifdef TVM_ATTN_TIMELINE
+void tvm_attn_debug_set_timeline(unsigned long long* device_ptr) { g_timeline = device_ptr; }
 #endif
 
 }  // extern "C"
