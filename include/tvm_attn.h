@@ -53,8 +53,9 @@ typedef struct {
 
 /*
  * Bytes of device scratch the forward (is_bwd == 0) or backward (is_bwd != 0) call needs for these
- * parameters.  The forward needs none.  The backward keeps two floats per query row there (the row
- * sums of App. C "Step 1", in the form rowsum(dtO*O) and rowsum(dO*O) + rowsum(dtO*tO)).
+ * parameters.  The forward needs none.  The backward keeps three floats per query row there (the row
+ * sums of App. C "Step 1", in the form rowsum(dtO*O) and rowsum(dO*O) + rowsum(dtO*tO), and lse in
+ * log2 units).
  * Returns 0 for invalid parameters.
  */
 size_t tvm_attn_jvp_workspace_bytes(const tvm_attn_params* p, int is_bwd);

@@ -1,0 +1,605 @@
+// Backward kernels of attention with a Jacobian-vector product on sm_100a (tcgen05 + TMEM + TMA),
+// for padded head dims up to 80 (d = 72 runs as 80).  Three passes share one skeleton (App. C
+// "Multi-step backward pass" with the standard attention backward for dO summed in):
+//
+//   pass  owner rows  stream rows  score accumulators (128 x BC fp32)                   bf16 operands A0, A1   acc0, acc1 (128 x d)
+//   DV    keys        queries      S^T = K Q^T, Sd^T = tK Q^T + K tQ^T                    P^T, (P Nn)^T          dtV, dV          (step 6)
+//   DK    keys        queries      S^T, Sd^T, D^T = V Hc^T, X^T = tV Hc^T + V G^T        W^T, dA^T              dtK/alpha, dK/alpha   (steps 2, 4)
+//   DQ    queries     keys         S, Sd, D = Hc V^T, X = G V^T + Hc tV^T                 W, dA                  dtQ/alpha, dQ/alpha   (steps 3, 5)
+//
+// with P = 2^(c2 S - lse2), Nn = alpha Sd - mu, W = P (D - Sigma1), dA = P (X - c) + W Nn, and
+//   acc0 += A0 B0,  acc1 += A1 B0 + A0 B1      (B0, B1 = Hc, G | Q, tQ | K, tK).
+//
+// A CTA owns 128 owner rows of one head and streams the other side in tiles of BC rows (64 for DV,
+// 32 for DK and DQ, whose four score accumulators need twice the tensor-memory columns).
+//
+// What is where
+//   * The owner operands of the first score pair (K, tK or Q, tQ) are written once into tensor memory
+//     as bf16 A operands: with A in tensor memory a 128 x N x 16 MMA runs at full rate for N >= 32,
+//     while with A in shared memory it is bound by the shared-memory port (N = 32: 40 clk instead of 16).
+//     The owner operands of the second score pair (V, tV or Hc, G) stay in shared memory: tensor
+//     memory has no room for them next to two score buffers.
+//   * Score accumulators are double-buffered; the bf16 operands A0, A1 are written back over the
+//     columns of the first two accumulators and consumed from tensor memory.
+//   * 16 element-wise warps: warp w works on TMEM lane quadrant w % 4 (32 owner rows) and on the
+//     slice w / 4 (BC / 4 columns) of every tile.  Nothing is exchanged between them.
+//   * Streamed columns 0..63 arrive by TMA; columns from 64 on are 16-byte asynchronous copies (a
+//     64-column box hanging over the end of a 144-byte row would read the next row from L2 for nothing).
+//   * Per-query statistics of the transposed passes (DV, DK) are staged in shared memory by warp 3.
+//
+// Every wait on an mbarrier is bounded; when one gives up the block records a time-out status and
+// all roles leave their loops.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "sm100_ptx.cuh"
+
+namespace tvm_attn {
+
+enum : int { BWD_DV = 0, BWD_DK = 1, BWD_DQ = 2 };
+
+constexpr int BWD_THREADS = 640;  // 4 control warps + 16 element-wise warps
+constexpr int BWD_ROWS = 128;     // owner rows per CTA
+constexpr int BWD_STATS_STAGES = 8;  // ring of per-query statistics tiles
+constexpr int BWD_STATS_LAG = 3;     // statistics copies in flight
+constexpr uint64_t BWD_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;
+
+struct BwdParams {
+    int N, d, BH;
+    float alpha;      // softmax scale
+    float c2;         // alpha * log2(e)
+    float out_scale;  // factor applied to acc0 / acc1 in the epilogue
+    const __nv_bfloat16* own[4];  // owner tensors X0..X3 (X2, X3 unused by DV)
+    const __nv_bfloat16* strm[4]; // streamed tensors: E ring (0, 1), L ring (2, 3)
+    __nv_bfloat16* out0;          // acc0 destination: dtV | dtK | dtQ
+    __nv_bfloat16* out1;          // acc1 destination: dV | dK | dQ
+    const float* lse2;  // lse * log2(e), written by the row-sums pre-pass
+    const float* mu;
+    const float* sig1;  // rowsum(dtO * O)
+    const float* cvec;  // rowsum(dO * O) + rowsum(dtO * tO)
+    int* status;        // device status word; non-zero makes the kernel a no-op
+    unsigned long long* tl;  // timeline builds only: clock stamps of CTA 0
+};
+
+#ifdef TVM_ATTN_TIMELINE
+#define BTL_STAMP(role, j, ev)                                                                         \
+    do {                                                                                                \
+        if (p.tl && blockIdx.x == 0 && (j) < 64) {                                                      \
+            unsigned long long t_;                                                                      \
+            asm volatile("mov.u64 %0, %clock64;" : "=l"(t_));                                          \
+            p.tl[((role) * 64 + (j)) * 8 + (ev)] = t_;                                                  \
+        }                                                                                               \
+    } while (0)
+#else
+#define BTL_STAMP(role, j, ev) do {} while (0)
+#endif
+
+template <int MODE, int DP>
+struct BwdCfg {
+    static_assert(DP % 16 == 0 && DP >= 16 && DP <= 80, "padded head dim must be 16..80");
+    static constexpr int NPAIR = MODE == BWD_DV ? 1 : 2;   // score pairs
+    static constexpr int BC = NPAIR == 1 ? 64 : 32;        // stream rows per tile
+    static constexpr int CW = BC / 4;                      // columns per element-wise warp
+    static constexpr bool TRANSPOSED = MODE != BWD_DQ;     // owner rows are keys
+    static constexpr int KS = DP / 16;
+    static constexpr int NA = DP > 64 ? 2 : 1;             // 64-column swizzle atoms per row
+    static constexpr int OWN_BYTES = NA * BWD_ROWS * 128;  // one owner tensor in shared memory
+    static constexpr int NOWN_SMEM = NPAIR == 2 ? 2 : 0;
+    static constexpr int ST_BYTES = NA * BC * 128;         // one streamed tensor tile
+    static constexpr int SE = NA == 1 ? 4 : (NPAIR == 1 ? 3 : 4);
+    static constexpr int SL = SE;
+    static constexpr int TILE_BYTES = NOWN_SMEM * OWN_BYTES + (SE + SL) * 2 * ST_BYTES;
+    static constexpr int FULL_COUNT = NA;                  // TMA issuer (+ the warp copying columns >= 64)
+    // which ring holds what: the E ring is released after the score MMAs, the L ring after the output MMAs.
+    // DV: E = (Q, tQ) score operands, L = (Hc, G) output operands.
+    // DK, DQ: E = second-pair score operands (Hc, G | V, tV), L = first-pair score operands that are also
+    // the output operands (Q, tQ | K, tK).
+    // barrier slots
+    static constexpr int B_EFULL = 0;
+    static constexpr int B_EEMPTY = B_EFULL + SE;
+    static constexpr int B_LFULL = B_EEMPTY + SE;
+    static constexpr int B_LEMPTY = B_LFULL + SL;
+    static constexpr int B_SFULL = B_LEMPTY + SL;
+    static constexpr int B_PREADY = B_SFULL + 2;
+    static constexpr int B_FINAL = B_PREADY + 2;
+    static constexpr int B_QREADY = B_FINAL + 1;
+    static constexpr int B_OWNER = B_QREADY + 1;
+    static constexpr int B_STFULL = B_OWNER + 1;
+    static constexpr int B_STEMPTY = B_STFULL + BWD_STATS_STAGES;
+    static constexpr int NBARS = B_STEMPTY + BWD_STATS_STAGES;
+    static_assert(NBARS <= 48, "barrier table too small");
+    static constexpr int STATS_FLOATS = BWD_STATS_STAGES * 4 * 64;
+    static constexpr int MISC_BYTES = 48 * 8 + 64 + STATS_FLOATS * 4;
+    static constexpr int SMEM_BYTES = TILE_BYTES + MISC_BYTES + 1024 /*alignment slack*/;
+    // TMEM columns: accumulators, the bf16 owner operands X0, X1 in the gaps behind them, two score buffers
+    static constexpr int COL_ACC0 = 0, COL_X0 = DP, COL_ACC1 = 128, COL_X1 = 128 + DP, COL_SCORE = 256;
+    static constexpr int SCORE_BUF_COLS = 2 * NPAIR * BC;
+    static_assert(DP + DP / 2 <= 128, "operand does not fit behind its accumulator");
+    static_assert(COL_SCORE + 2 * SCORE_BUF_COLS <= 512, "TMEM over-subscribed");
+};
+
+// One element of the backward element-wise stage.  s, ts (and d, x for DK/DQ) are the raw score
+// accumulators; lse2 = lse * log2(e); returns the two bf16-bound operand values.
+template <int MODE>
+__device__ __forceinline__ void bwd_element(const BwdParams& p, float s, float ts, float dd, float xx, float lse2,
+                                            float mu, float sg, float cv, float& a0, float& a1) {
+    const float P = ptx::ex2(fmaf(s, p.c2, -lse2));
+    const float Nn = fmaf(p.alpha, ts, -mu);
+    if (MODE == BWD_DV) {
+        a0 = P;
+        a1 = P * Nn;
+    } else {
+        const float W = P * (dd - sg);
+        a0 = W;
+        a1 = fmaf(P, xx - cv, W * Nn);
+    }
+}
+
+// Element-wise warps of the backward passes: `w` in 0..15.
+template <int MODE, int DP>
+__device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tmem_base, uint32_t bar0,
+                                                volatile int* abort_flag, const float* stats, int w, int lane, int bh,
+                                                int row0, int T) {
+    using C = BwdCfg<MODE, DP>;
+    constexpr int BC = C::BC, KS = C::KS, NPAIR = C::NPAIR;
+    constexpr int SLICES = BC / 16;     // 16-column slices per tile = k-steps of the output GEMMs
+    constexpr int GROUPS = 4 / SLICES;  // warp groups that alternate over the tiles
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
+    const int q = w & 3, slot = w >> 2;
+    const int sl = slot % SLICES, grp = slot / SLICES;
+    const int row = q * 32 + lane;  // owner row inside the CTA tile
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    const bool row_valid = row0 + row < p.N;
+    const size_t grow = (size_t)bh * p.N + row0 + row;
+
+    // ---- owner rows of X0 and X1 -> bf16 operands in tensor memory (k-step kk at 8 packed columns)
+    for (int ch = slot; ch < 2 * KS; ch += 4) {
+        const bool second = ch >= KS;
+        const int kk = second ? ch - KS : ch;
+        const __nv_bfloat16* src = p.own[second ? 1 : 0] + grow * p.d + 16 * kk;
+        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+        if (row_valid && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
+        if (row_valid && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
+        const uint32_t r[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        ptx::tmem_st8(lane_addr + (second ? C::COL_X1 : C::COL_X0) + 8 * kk, r);
+    }
+    ptx::tmem_wait_st();
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+
+    float r_lse2 = CUDART_INF_F, r_mu = 0.f, r_s1 = 0.f, r_cv = 0.f;  // per-row statistics (DQ)
+    if (MODE == BWD_DQ && row_valid) {
+        r_lse2 = p.lse2[grow];
+        r_mu = p.mu[grow];
+        r_s1 = p.sig1[grow];
+        r_cv = p.cvec[grow];
+    }
+    bool ok = true;
+    for (int j = grp; j < T; j += GROUPS) {
+        const int b = j & 1;
+        if (!ptx::mbar_wait(bar(C::B_SFULL + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        const float* st = stats + (j % BWD_STATS_STAGES) * 4 * 64 + 16 * sl;
+        if (C::TRANSPOSED)
+            if (!ptx::mbar_wait(bar(C::B_STFULL + j % BWD_STATS_STAGES), (j / BWD_STATS_STAGES) & 1, abort_flag,
+                                BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 0);
+        const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
+        const int key0 = j * BC + 16 * sl;  // first stream row of this slice
+        if (NPAIR == 1) {
+            uint32_t s1[16], s2[16];
+            ptx::tmem_ld16(sbase, s1);
+            ptx::tmem_ld16(sbase + BC, s2);
+            ptx::tmem_wait_ld();
+            uint32_t pa0[8], pa1[8];
+#pragma unroll
+            for (int c4 = 0; c4 < 16; c4 += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
+                const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
+                const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
+                float a0[4], a1[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    bwd_element<MODE>(p, __uint_as_float(s1[c4 + e]), __uint_as_float(s2[c4 + e]), 0.f, 0.f, lv[e], mv[e], 0.f,
+                                      0.f, a0[e], a1[e]);
+                pa0[c4 >> 1] = ptx::pack_bf16(a0[0], a0[1]);
+                pa0[(c4 >> 1) + 1] = ptx::pack_bf16(a0[2], a0[3]);
+                pa1[c4 >> 1] = ptx::pack_bf16(a1[0], a1[1]);
+                pa1[(c4 >> 1) + 1] = ptx::pack_bf16(a1[2], a1[3]);
+            }
+            // operand of k-step sl (16 stream rows) sits at column 16*sl of the accumulator it replaces
+            ptx::tmem_st8(sbase, pa0);
+            ptx::tmem_st8(sbase + BC, pa1);
+        } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t s1[8], s2[8], s3[8], s4[8];
+                ptx::tmem_ld8(sbase + 8 * h, s1);
+                ptx::tmem_ld8(sbase + BC + 8 * h, s2);
+                ptx::tmem_ld8(sbase + 2 * BC + 8 * h, s3);
+                ptx::tmem_ld8(sbase + 3 * BC + 8 * h, s4);
+                ptx::tmem_wait_ld();
+                uint32_t pa0[4], pa1[4];
+#pragma unroll
+                for (int c4 = 0; c4 < 8; c4 += 4) {
+                    float lv[4], mv[4], gv[4], cvv[4];
+                    if (C::TRANSPOSED) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(st + 8 * h + c4);
+                        const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + 8 * h + c4);
+                        const float4 g4 = *reinterpret_cast<const float4*>(st + 128 + 8 * h + c4);
+                        const float4 c44 = *reinterpret_cast<const float4*>(st + 192 + 8 * h + c4);
+                        lv[0] = l4.x; lv[1] = l4.y; lv[2] = l4.z; lv[3] = l4.w;
+                        mv[0] = m4.x; mv[1] = m4.y; mv[2] = m4.z; mv[3] = m4.w;
+                        gv[0] = g4.x; gv[1] = g4.y; gv[2] = g4.z; gv[3] = g4.w;
+                        cvv[0] = c44.x; cvv[1] = c44.y; cvv[2] = c44.z; cvv[3] = c44.w;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            lv[e] = (key0 + 8 * h + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
+                            mv[e] = r_mu; gv[e] = r_s1; cvv[e] = r_cv;
+                        }
+                    }
+                    float a0[4], a1[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        bwd_element<MODE>(p, __uint_as_float(s1[c4 + e]), __uint_as_float(s2[c4 + e]),
+                                          __uint_as_float(s3[c4 + e]), __uint_as_float(s4[c4 + e]), lv[e], mv[e], gv[e],
+                                          cvv[e], a0[e], a1[e]);
+                    pa0[c4 >> 1] = ptx::pack_bf16(a0[0], a0[1]);
+                    pa0[(c4 >> 1) + 1] = ptx::pack_bf16(a0[2], a0[3]);
+                    pa1[c4 >> 1] = ptx::pack_bf16(a1[0], a1[1]);
+                    pa1[(c4 >> 1) + 1] = ptx::pack_bf16(a1[2], a1[3]);
+                }
+                // half h of the k-step's operand: 4 packed columns.  They overwrite accumulator columns of
+                // this warp's own slice that it has already read.
+                ptx::tmem_st4(sbase + 4 * h, pa0);
+                ptx::tmem_st4(sbase + BC + 4 * h, pa1);
+            }
+        }
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);
+        if (lane == 0) {
+            ptx::mbar_arrive(bar(C::B_PREADY + b));
+            if (C::TRANSPOSED) ptx::mbar_arrive(bar(C::B_STEMPTY + j % BWD_STATS_STAGES));
+        }
+    }
+    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+    if (ok) {
+        ptx::tc_fence_after_sync();
+        __nv_bfloat16* p0 = p.out0 + grow * p.d;
+        __nv_bfloat16* p1 = p.out1 + grow * p.d;
+        for (int ch = slot; ch < KS; ch += 4) {
+            uint32_t x0[16], x1[16];
+            ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, x0);
+            ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, x1);
+            ptx::tmem_wait_ld();
+            uint32_t q0[8], q1[8];
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) {
+                q0[c >> 1] = ptx::pack_bf16(__uint_as_float(x0[c]) * p.out_scale, __uint_as_float(x0[c + 1]) * p.out_scale);
+                q1[c >> 1] = ptx::pack_bf16(__uint_as_float(x1[c]) * p.out_scale, __uint_as_float(x1[c + 1]) * p.out_scale);
+            }
+            if (row_valid) {
+                *reinterpret_cast<uint4*>(p0 + 16 * ch) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
+                *reinterpret_cast<uint4*>(p1 + 16 * ch) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
+                if (16 * ch + 8 < p.d) {
+                    *reinterpret_cast<uint4*>(p0 + 16 * ch + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
+                    *reinterpret_cast<uint4*>(p1 + 16 * ch + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
+                }
+            }
+        }
+    }
+}
+
+template <int MODE, int DP>
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant__ CUtensorMap tm_s1,
+               const __grid_constant__ CUtensorMap tm_s2, const __grid_constant__ CUtensorMap tm_s3,
+               const __grid_constant__ CUtensorMap tm_o2, const __grid_constant__ CUtensorMap tm_o3,
+               const BwdParams p) {
+    using C = BwdCfg<MODE, DP>;
+    constexpr int BC = C::BC, KS = C::KS, NA = C::NA, SE = C::SE, SL = C::SL, NPAIR = C::NPAIR;
+    if (*reinterpret_cast<volatile int*>(p.status) != 0) return;  // an earlier kernel timed out
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t own_base = ptx::smem_u32(smem);
+    const uint32_t e_base = own_base + C::NOWN_SMEM * C::OWN_BYTES;
+    const uint32_t l_base = e_base + SE * 2 * C::ST_BYTES;
+    uint8_t* misc = smem + C::TILE_BYTES;
+    const uint32_t bar0 = ptx::smem_u32(misc);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 48 * 8 + 16);
+    float* stats = reinterpret_cast<float*>(misc + 48 * 8 + 64);  // [stage][4][64]
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row_tiles = (p.N + BWD_ROWS - 1) / BWD_ROWS;
+    const int bh = blockIdx.x / row_tiles;
+    const int row0 = (blockIdx.x - bh * row_tiles) * BWD_ROWS;
+    const int T = (p.N + BC - 1) / BC;  // stream tiles
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
+        for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(bar(C::B_SFULL + b), 1);
+            ptx::mbar_init(bar(C::B_PREADY + b), BC / 4);  // one arrival per warp working on a tile
+        }
+        ptx::mbar_init(bar(C::B_FINAL), 1);
+        ptx::mbar_init(bar(C::B_QREADY), 16);
+        ptx::mbar_init(bar(C::B_OWNER), C::FULL_COUNT);
+        for (int s = 0; s < BWD_STATS_STAGES; ++s) {
+            ptx::mbar_init(bar(C::B_STFULL + s), 1);
+            ptx::mbar_init(bar(C::B_STEMPTY + s), BC / 4);
+        }
+        ptx::fence_mbar_init();
+    }
+    if (NA == 2) {
+        // Second swizzle atom of every tile: the 16-byte chunk behind the copied columns must read as zero
+        // (it pads d to a multiple of 16) and is never written again.  Logical chunk k of row r sits at
+        // physical chunk k ^ (r & 7).
+        if (((p.d - 64) >> 3) < 2) {
+            for (int i = threadIdx.x; i < C::NOWN_SMEM * BWD_ROWS; i += BWD_THREADS) {
+                const int t = i / BWD_ROWS, r = i - t * BWD_ROWS;
+                uint8_t* atom2 = smem + t * C::OWN_BYTES + BWD_ROWS * 128;
+                *reinterpret_cast<uint4*>(atom2 + r * 128 + ((1 ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            }
+            for (int i = threadIdx.x; i < (SE + SL) * 2 * BC; i += BWD_THREADS) {
+                const int t = i / BC, r = i - t * BC;
+                uint8_t* atom2 = smem + C::NOWN_SMEM * C::OWN_BYTES + t * C::ST_BYTES + BC * 128;
+                *reinterpret_cast<uint4*>(atom2 + r * 128 + ((1 ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            }
+            ptx::fence_proxy_async_smem();
+        }
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) BTL_STAMP(3, 0, 0);
+
+    // shared-memory address of tile j of streamed tensor t (0, 1: E ring; 2, 3: L ring)
+    auto tile_addr = [&](int t, int j) -> uint32_t {
+        return t < 2 ? e_base + ((j % SE) * 2 + t) * C::ST_BYTES : l_base + ((j % SL) * 2 + (t - 2)) * C::ST_BYTES;
+    };
+
+    if (warp == 0 || warp == 2) {
+        // ------------------------------------------------------------------ producers: warp 0 feeds the E
+        // ring (and loads the shared-memory owner tiles first), warp 2 the L ring.  Lane 0 issues the TMA
+        // boxes of columns 0..63; all lanes copy the columns from 64 on, 16 bytes per row and chunk, and
+        // signal them one tile later so that two tiles of copies are in flight.
+        const int ring = warp >> 1;
+        const int S = ring == 0 ? SE : SL;
+        const int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
+        const CUtensorMap* maps[2] = {ring == 0 ? &tm_s0 : &tm_s2, ring == 0 ? &tm_s1 : &tm_s3};
+        const __nv_bfloat16* srcs[2] = {p.strm[2 * ring], p.strm[2 * ring + 1]};
+        const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
+        if (NPAIR == 2 && ring == 0) {
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
+                ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
+                ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
+            }
+            if constexpr (NA == 2) {
+                for (int i = lane; i < 2 * BWD_ROWS * ntail; i += 32) {
+                    const int t = i / (BWD_ROWS * ntail), rem = i - t * (BWD_ROWS * ntail);
+                    const int r = rem / ntail, k = rem - r * ntail;
+                    const bool v = row0 + r < p.N;
+                    const __nv_bfloat16* src = p.own[2 + t] + ((size_t)bh * p.N + (v ? row0 + r : 0)) * p.d + 64 + 8 * k;
+                    ptx::cp_async_16(own_base + t * C::OWN_BYTES + BWD_ROWS * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+                }
+                ptx::cp_async_commit();
+                ptx::cp_async_wait<0>();
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+            }
+        }
+        bool ok = true;
+        for (int j = 0; j < T; ++j) {
+            const int s = j % S, ph = (j / S) & 1;
+            ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
+            if (!ok) break;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
+                for (int t = 0; t < 2; ++t) ptx::tma_load_3d(tile_addr(2 * ring + t, j), maps[t], bar(b_full + s), 0, j * BC, bh);
+            }
+            if constexpr (NA == 2) {
+                for (int i = lane; i < 2 * BC * ntail; i += 32) {
+                    const int t = i / (BC * ntail), rem = i - t * (BC * ntail);
+                    const int r = rem / ntail, k = rem - r * ntail;
+                    const int grow = j * BC + r;
+                    const bool v = grow < p.N;
+                    const __nv_bfloat16* src = srcs[t] + ((size_t)bh * p.N + (v ? grow : 0)) * p.d + 64 + 8 * k;
+                    ptx::cp_async_16(tile_addr(2 * ring + t, j) + BC * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+                }
+                ptx::cp_async_commit();
+                if (j > 0) {
+                    ptx::cp_async_wait<1>();
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(b_full + (j - 1) % S));
+                }
+            }
+        }
+        if (NA == 2 && ok) {
+            ptx::cp_async_wait<0>();
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(b_full + (T - 1) % S));
+        }
+        if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer: the whole warp runs
+        // the loop in converged control flow; one elected lane issues (see mma_ts_elect)
+        constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
+        constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
+        const uint32_t ax0 = tb + C::COL_X0, ax1 = tb + C::COL_X1;
+        // owner tiles in shared memory (second score pair), K-major A operands
+        const uint64_t o2d = ptx::smem_desc_sw128(own_base, 16, 1024);
+        const uint64_t o3d = ptx::smem_desc_sw128(own_base + C::OWN_BYTES, 16, 1024);
+        auto issue_scores = [&](int j) -> bool {
+            const int b = j & 1;
+            if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (NPAIR == 2)
+                if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            ptx::tc_fence_after_sync();
+            if (lane == 0) BTL_STAMP(0, j, 0);
+            // first-pair stream operands Y0, Y1: E ring for DV, L ring for DK/DQ; K-major B
+            const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(NPAIR == 1 ? 0 : 2, j), 16, 1024);
+            const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(NPAIR == 1 ? 1 : 3, j), 16, 1024);
+            const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {  // S = X0 Y0^T
+                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                ptx::mma_ts_elect(dS, ax0 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+            }
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {  // Sd = X1 Y0^T
+                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                ptx::mma_ts_elect(dT, ax1 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+            }
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {  // Sd += X0 Y1^T
+                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                ptx::mma_ts_elect(dT, ax0 + 8 * kk, y1 + off, idesc_s, 1u);
+            }
+            if (NPAIR == 2) {
+                const uint64_t y2 = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
+                const uint64_t y3 = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
+                const uint32_t dD = dS + 2 * BC, dX = dS + 3 * BC;
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {  // D = X2 Y2^T
+                    const uint64_t offa = (uint64_t)(((kk >> 2) * BWD_ROWS * 128 + (kk & 3) * 32) >> 4);
+                    const uint64_t offb = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ss_elect(dD, o2d + offa, y2 + offb, idesc_s, kk > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {  // X = X3 Y2^T
+                    const uint64_t offa = (uint64_t)(((kk >> 2) * BWD_ROWS * 128 + (kk & 3) * 32) >> 4);
+                    const uint64_t offb = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ss_elect(dX, o3d + offa, y2 + offb, idesc_s, kk > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {  // X += X2 Y3^T
+                    const uint64_t offa = (uint64_t)(((kk >> 2) * BWD_ROWS * 128 + (kk & 3) * 32) >> 4);
+                    const uint64_t offb = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ss_elect(dX, o2d + offa, y3 + offb, idesc_s, 1u);
+                }
+            }
+            ptx::mma_commit_elect(bar(C::B_SFULL + b));
+            ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+            if (lane == 0) BTL_STAMP(0, j, 1);
+            return true;
+        };
+        auto issue_outputs = [&](int j) -> bool {
+            const int b = j & 1;
+            if (NPAIR == 1)
+                if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (lane == 0) BTL_STAMP(0, j, 2);
+            if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            ptx::tc_fence_after_sync();
+            if (lane == 0) BTL_STAMP(0, j, 3);
+            const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
+            // MN-major B (the L ring): atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
+            const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
+            const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+            const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+#pragma unroll
+            for (int u = 0; u < BC / 16; ++u) {
+                const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                ptx::mma_ts_elect(acc0, a0 + 16 * u, b0 + off, idesc_o, acc);   // acc0 += A0 B0
+                ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc_o, acc);   // acc1 += A1 B0
+                ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, 1u);    // acc1 += A0 B1
+            }
+            ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+            if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+            if (lane == 0) BTL_STAMP(0, j, 4);
+            return true;
+        };
+        bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+        if (ok && NPAIR == 2) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+        ptx::tc_fence_after_sync();
+        if (ok) ok = issue_scores(0);
+        for (int j = 0; ok && j < T; ++j) {
+            if (j + 1 < T) ok = issue_scores(j + 1);
+            if (ok) ok = issue_outputs(j);
+        }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ per-query statistics (transposed passes):
+        // lse2, mu (and Sigma1, c for DK) of the tile's queries, copied asynchronously into a ring so that
+        // their latency (about a microsecond per global load) stays off the tile loop.
+        if (C::TRANSPOSED) {
+            const size_t srow = (size_t)bh * p.N;
+            const float* src_stat[4] = {p.lse2, p.mu, p.sig1, p.cvec};
+            if ((p.N & 3) == 0) {
+                constexpr int CPS = BC / 4;  // 16-byte chunks per statistic and tile; 32 chunks per tile in all
+                const int stat = lane / CPS, chunk = lane - stat * CPS;
+                const float* src = src_stat[stat] + srow + 4 * chunk;
+                bool ok = true;
+                for (int j = 0; j < T; ++j) {
+                    const int s = j % BWD_STATS_STAGES, ph = (j / BWD_STATS_STAGES) & 1;
+                    ok = ptx::mbar_wait_warp(bar(C::B_STEMPTY + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    if (!ok) break;
+                    const bool v = j * BC + 4 * chunk < p.N;  // queries beyond N read as zero: their B rows are zero too
+                    ptx::cp_async_16(ptx::smem_u32(stats + s * 4 * 64 + stat * 64 + 4 * chunk), src + (v ? j * BC : 0), v ? 16u : 0u);
+                    ptx::cp_async_commit();
+                    if (j >= BWD_STATS_LAG) {
+                        ptx::cp_async_wait<BWD_STATS_LAG>();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(C::B_STFULL + (j - BWD_STATS_LAG) % BWD_STATS_STAGES));
+                    }
+                }
+                ptx::cp_async_wait<0>();
+                __syncwarp();
+                if (ok && lane == 0)
+                    for (int j = (T > BWD_STATS_LAG ? T - BWD_STATS_LAG : 0); j < T; ++j)
+                        ptx::mbar_arrive(bar(C::B_STFULL + j % BWD_STATS_STAGES));
+            } else {
+                // rows of the statistics are not 16-byte aligned for this N: plain loads, one tile at a time
+                for (int j = 0; j < T; ++j) {
+                    const int s = j % BWD_STATS_STAGES, ph = (j / BWD_STATS_STAGES) & 1;
+                    if (!ptx::mbar_wait_warp(bar(C::B_STEMPTY + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS)) break;
+                    float* st = stats + s * 4 * 64;
+                    for (int c = lane; c < BC; c += 32) {
+                        const int i = j * BC + c;
+                        const bool v = i < p.N;
+#pragma unroll
+                        for (int k = 0; k < 2 * NPAIR; ++k) st[k * 64 + c] = v ? src_stat[k][srow + i] : 0.f;
+                    }
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(C::B_STFULL + s));
+                }
+            }
+        }
+    } else {
+        bwd_elementwise<MODE, DP>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, bh, row0, T);
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0) BTL_STAMP(3, 0, 1);
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, 1);
+}
+
+}  // namespace tvm_attn

@@ -162,8 +162,8 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
 template <typename T>
 __global__ void __launch_bounds__(256)
 bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* __restrict__ O,
-                   const T* __restrict__ tO, float* __restrict__ sig1, float* __restrict__ cvec,
-                   long long rows, int d) {
+                   const T* __restrict__ tO, const float* __restrict__ lse, float* __restrict__ sig1,
+                   float* __restrict__ cvec, float* __restrict__ lse2, long long rows, int d) {
     const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -178,7 +178,7 @@ bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* _
     }
     s1 = warp_sum(s1);
     cc = warp_sum(cc);
-    if (lane == 0) { sig1[row] = s1; cvec[row] = cc; }
+    if (lane == 0) { sig1[row] = s1; cvec[row] = cc; lse2[row] = lse[row] * 1.4426950408889634f; }
 }
 
 // The four per-pair quantities of the backward from the six dot products of a (query, key) pair.

@@ -12,12 +12,16 @@
 #include <mutex>
 
 #include "dual_attn_sm100.cuh"
+#include "jvp_bwd_sm100.cuh"
 #include "jvp_fwd_sm100.cuh"
 #include "simt_kernels.cuh"
 
 namespace tvm_attn {
 
 static std::atomic<uint64_t> g_launches{0};
+#ifdef TVM_ATTN_TIMELINE
+static unsigned long long* g_timeline = nullptr;  // clock stamps of CTA 0 (timeline builds only)
+#endif
 __device__ int g_status_word = 0;  // raised by a tensor-core kernel whose bounded wait ran out
 
 // Optional per-kernel timing: events recorded around each launch of the most recent call.
@@ -86,13 +90,13 @@ static int simt_fwd(const Shape& s, const void* Q, const void* K, const void* V,
 }
 
 template <typename T>
-static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const void* O, const void* tO, float* sig1,
-                          float* cvec, cudaStream_t st) {
+static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const void* O, const void* tO, const float* lse,
+                          float* sig1, float* cvec, float* lse2, cudaStream_t st) {
     const long long rows = s.BH * s.N;
     const unsigned grid = (unsigned)((rows + 7) / 8);
     g_prof.before(st);
-    bwd_rowsums_kernel<T><<<grid, 256, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, sig1, cvec, rows,
-                                                s.d);
+    bwd_rowsums_kernel<T><<<grid, 256, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, lse, sig1, cvec,
+                                                lse2, rows, s.d);
     g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
@@ -217,11 +221,46 @@ static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams
     return cuda_status(cudaGetLastError());
 }
 
+// One backward pass for padded head dims up to 80 (jvp_bwd_sm100.cuh).  own: X0..X3; strm: E ring (0, 1), L ring (2, 3).
+template <int MODE, int DP>
+static int launch_bwd_pass(const Shape& s, const void* const own[4], const void* const strm[4], BwdParams prm, cudaStream_t st) {
+    using C = BwdCfg<MODE, DP>;
+    CUtensorMap ms[4], mo[2];
+    for (int t = 0; t < 4; ++t) {
+        const int rc = make_tmap(&ms[t], strm[t], s, C::BC);
+        if (rc != TVM_ATTN_OK) return rc;
+        prm.strm[t] = static_cast<const __nv_bfloat16*>(strm[t]);
+        prm.own[t] = static_cast<const __nv_bfloat16*>(own[t]);
+    }
+    for (int t = 0; t < 2; ++t) {
+        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? 2 + t : t], s, BWD_ROWS);
+        if (rc != TVM_ATTN_OK) return rc;
+    }
+    auto kern = jvp_bwd_kernel<MODE, DP>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        return TVM_ATTN_CUDA_ERROR;
+    const long long grid = s.BH * ((s.N + BWD_ROWS - 1) / BWD_ROWS);
+    g_prof.before(st);
+    kern<<<(unsigned)grid, BWD_THREADS, C::SMEM_BYTES, st>>>(ms[0], ms[1], ms[2], ms[3], mo[0], mo[1], prm);
+    g_prof.after(st);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
+template <int MODE>
+static int launch_bwd_pass_dp(const Shape& s, const void* const own[4], const void* const strm[4], const BwdParams& prm,
+                              cudaStream_t st) {
+    switch (s.dp) {
+        case 16: return launch_bwd_pass<MODE, 16>(s, own, strm, prm, st);
+        case 32: return launch_bwd_pass<MODE, 32>(s, own, strm, prm, st);
+        case 48: return launch_bwd_pass<MODE, 48>(s, own, strm, prm, st);
+        case 64: return launch_bwd_pass<MODE, 64>(s, own, strm, prm, st);
+        default: return launch_bwd_pass<MODE, 80>(s, own, strm, prm, st);
+    }
+}
+
 #ifdef TVM_ATTN_DEBUG_DUMP
 static float* g_debug_dump = nullptr;
-#endif
-#ifdef TVM_ATTN_TIMELINE
-static unsigned long long* g_timeline = nullptr;  // clock stamps of CTA 0 (timeline builds only)
 #endif
 
 static TcParams base_params(const Shape& s, int* status) {
@@ -248,7 +287,7 @@ size_t tvm_attn_jvp_workspace_bytes(const tvm_attn_params* p, int is_bwd) {
     Shape s;
     if (check_params(p, &s) != TVM_ATTN_OK) return 0;
     if (!is_bwd) return 0;
-    return (size_t)2 * sizeof(float) * (size_t)s.BH * (size_t)s.N;
+    return (size_t)3 * sizeof(float) * (size_t)s.BH * (size_t)s.N;
 }
 
 int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, const void* V, const void* tQ,
@@ -311,18 +350,19 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     for (const void* x : ptrs)
         if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
     const size_t rows = (size_t)s.BH * (size_t)s.N;
-    if (workspace_bytes < 2 * sizeof(float) * rows) return TVM_ATTN_WORKSPACE_TOO_SMALL;
+    if (workspace_bytes < 3 * sizeof(float) * rows) return TVM_ATTN_WORKSPACE_TOO_SMALL;
     float* sig1 = static_cast<float*>(workspace);
     float* cvec = sig1 + rows;
+    float* lse2 = cvec + rows;  // lse * log2(e)
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     g_prof.begin_call();
     if (s.simt) {
         if (s.fp32) {
-            rc = launch_rowsums<float>(s, dO, dtO, O, tO, sig1, cvec, st);
+            rc = launch_rowsums<float>(s, dO, dtO, O, tO, lse, sig1, cvec, lse2, st);
             if (rc != TVM_ATTN_OK) return rc;
             return simt_bwd<float>(s, Q, K, V, tQ, tK, tV, lse, mu, dO, dtO, sig1, cvec, dQ, dK, dV, dtQ, dtK, dtV, st);
         }
-        rc = launch_rowsums<__nv_bfloat16>(s, dO, dtO, O, tO, sig1, cvec, st);
+        rc = launch_rowsums<__nv_bfloat16>(s, dO, dtO, O, tO, lse, sig1, cvec, lse2, st);
         if (rc != TVM_ATTN_OK) return rc;
         return simt_bwd<__nv_bfloat16>(s, Q, K, V, tQ, tK, tV, lse, mu, dO, dtO, sig1, cvec, dQ, dK, dV, dtQ, dtK, dtV, st);
     }
@@ -330,8 +370,44 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     if (rc != TVM_ATTN_OK) return rc;
     int* status = status_word_ptr();
     if (!status) return TVM_ATTN_CUDA_ERROR;
-    rc = launch_rowsums<__nv_bfloat16>(s, dO, dtO, O, tO, sig1, cvec, st);
+    rc = launch_rowsums<__nv_bfloat16>(s, dO, dtO, O, tO, lse, sig1, cvec, lse2, st);
     if (rc != TVM_ATTN_OK) return rc;
+    if (s.dp <= 80) {
+        BwdParams b;
+        std::memset(&b, 0, sizeof b);
+        b.N = s.N; b.d = s.d; b.BH = (int)s.BH;
+        b.alpha = s.alpha; b.c2 = s.alpha * 1.4426950408889634f;
+        b.lse2 = lse2; b.mu = mu; b.sig1 = sig1; b.cvec = cvec; b.status = status;
+#ifdef TVM_ATTN_TIMELINE
+        b.tl = g_timeline;  // each pass gets its own third of the buffer (see below)
+#endif
+        {   // dtV = P^T Hc, dV = P^T G + (P*Nn)^T Hc : owner keys (K, tK); stream queries (Q, tQ | Hc, G)
+            BwdParams q = b; q.out_scale = 1.0f;
+            q.out0 = static_cast<__nv_bfloat16*>(dtV); q.out1 = static_cast<__nv_bfloat16*>(dV);
+            const void* own[4] = {K, tK, K, tK};
+            const void* strm[4] = {Q, tQ, dtO, dO};
+            rc = launch_bwd_pass_dp<BWD_DV>(s, own, strm, q, st);
+            if (rc != TVM_ATTN_OK) return rc;
+        }
+        {   // dtK = alpha W^T Q, dK = alpha (dA^T Q + W^T tQ) : owner keys (K, tK, V, tV); stream (Hc, G | Q, tQ)
+            BwdParams q = b; q.out_scale = s.alpha;
+            if (q.tl) q.tl += 4 * 64 * 8;
+            q.out0 = static_cast<__nv_bfloat16*>(dtK); q.out1 = static_cast<__nv_bfloat16*>(dK);
+            const void* own[4] = {K, tK, V, tV};
+            const void* strm[4] = {dtO, dO, Q, tQ};
+            rc = launch_bwd_pass_dp<BWD_DK>(s, own, strm, q, st);
+            if (rc != TVM_ATTN_OK) return rc;
+        }
+        {   // dtQ = alpha W K, dQ = alpha (dA K + W tK) : owner queries (Q, tQ, Hc, G); stream (V, tV | K, tK)
+            BwdParams q = b; q.out_scale = s.alpha;
+            if (q.tl) q.tl += 2 * 4 * 64 * 8;
+            q.out0 = static_cast<__nv_bfloat16*>(dtQ); q.out1 = static_cast<__nv_bfloat16*>(dQ);
+            const void* own[4] = {Q, tQ, dtO, dO};
+            const void* strm[4] = {V, tV, K, tK};
+            rc = launch_bwd_pass_dp<BWD_DQ>(s, own, strm, q, st);
+        }
+        return rc;
+    }
     TcParams prm = base_params(s, status);
     prm.lse = lse; prm.mu = mu; prm.sig1 = sig1; prm.cvec = cvec;
     {   // dtV = P^T Hc, dV = P^T G + (P*Nn)^T Hc : owner keys (K, tK), stream queries (Q, tQ | Hc, G)
