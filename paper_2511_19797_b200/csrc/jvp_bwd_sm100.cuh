@@ -82,17 +82,22 @@ template <int MODE, int DP>
 struct BwdCfg {
     static_assert(DP % 16 == 0 && DP >= 16 && DP <= 80, "padded head dim must be 16..80");
     static constexpr int NPAIR = MODE == BWD_DV ? 1 : 2;   // score pairs
-    static constexpr int BC = NPAIR == 1 ? 64 : 32;        // stream rows per tile
+    static constexpr int BC = 64;                          // stream rows per tile
     static constexpr int CW = BC / 4;                      // columns per element-wise warp
     static constexpr bool TRANSPOSED = MODE != BWD_DQ;     // owner rows are keys
     static constexpr int KS = DP / 16;
     static constexpr int NA = DP > 64 ? 2 : 1;             // 64-column swizzle atoms per row
-    static constexpr int OWN_BYTES = NA * BWD_ROWS * 128;  // one owner tensor in shared memory
+    // Tiles that are only ever read K-major (the shared-memory owner tensors and the E ring) keep the columns
+    // from 64 on in an unswizzled block behind the 64-column swizzle atom: [chunk][row][16 bytes], 32 bytes
+    // per row instead of a second 128-byte atom.  The L ring is also read MN-major by the output GEMMs, whose
+    // single N = DP operand needs one layout: two 128-byte-swizzled atoms.
+    static constexpr int OWN_BYTES = BWD_ROWS * 128 + (NA - 1) * BWD_ROWS * 32;  // one owner tensor in shared memory
     static constexpr int NOWN_SMEM = NPAIR == 2 ? 2 : 0;
-    static constexpr int ST_BYTES = NA * BC * 128;         // one streamed tensor tile
-    static constexpr int SE = NA == 1 ? 4 : (NPAIR == 1 ? 3 : 4);
-    static constexpr int SL = SE;
-    static constexpr int TILE_BYTES = NOWN_SMEM * OWN_BYTES + (SE + SL) * 2 * ST_BYTES;
+    static constexpr int EST_BYTES = BC * 128 + (NA - 1) * BC * 32;  // one E-ring tile
+    static constexpr int LST_BYTES = NA * BC * 128;                  // one L-ring tile
+    static constexpr int SE = NPAIR == 1 ? 4 : (NA == 1 ? 4 : 3);
+    static constexpr int SL = NA == 1 ? 4 : 3;
+    static constexpr int TILE_BYTES = NOWN_SMEM * OWN_BYTES + SE * 2 * EST_BYTES + SL * 2 * LST_BYTES;
     static constexpr int FULL_COUNT = NA;                  // TMA issuer (+ the warp copying columns >= 64)
     // which ring holds what: the E ring is released after the score MMAs, the L ring after the output MMAs.
     // DV: E = (Q, tQ) score operands, L = (Hc, G) output operands.
@@ -103,8 +108,8 @@ struct BwdCfg {
     static constexpr int B_EEMPTY = B_EFULL + SE;
     static constexpr int B_LFULL = B_EEMPTY + SE;
     static constexpr int B_LEMPTY = B_LFULL + SL;
-    static constexpr int B_SFULL = B_LEMPTY + SL;
-    static constexpr int B_PREADY = B_SFULL + 2;
+    static constexpr int B_SFULL = B_LEMPTY + SL;          // DV: per buffer.  DK/DQ: +0 (S, Sd) written, +1 (D, X) written
+    static constexpr int B_PREADY = B_SFULL + 2;           // DV: per buffer.  DK/DQ: +0 operands written, +1 (S, Sd) read
     static constexpr int B_FINAL = B_PREADY + 2;
     static constexpr int B_QREADY = B_FINAL + 1;
     static constexpr int B_OWNER = B_QREADY + 1;
@@ -117,9 +122,11 @@ struct BwdCfg {
     static constexpr int SMEM_BYTES = TILE_BYTES + MISC_BYTES + 1024 /*alignment slack*/;
     // TMEM columns: accumulators, the bf16 owner operands X0, X1 in the gaps behind them, two score buffers
     static constexpr int COL_ACC0 = 0, COL_X0 = DP, COL_ACC1 = 128, COL_X1 = 128 + DP, COL_SCORE = 256;
+    // DV: two buffers of (S | Sd).  DK, DQ: one buffer of (S | Sd | D | X), used in two phases.
     static constexpr int SCORE_BUF_COLS = 2 * NPAIR * BC;
+    static constexpr int NBUF = NPAIR == 1 ? 2 : 1;
     static_assert(DP + DP / 2 <= 128, "operand does not fit behind its accumulator");
-    static_assert(COL_SCORE + 2 * SCORE_BUF_COLS <= 512, "TMEM over-subscribed");
+    static_assert(COL_SCORE + NBUF * SCORE_BUF_COLS <= 512, "TMEM over-subscribed");
 };
 
 // One element of the backward element-wise stage.  s, ts (and d, x for DK/DQ) are the raw score
@@ -146,11 +153,9 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                                                 int row0, int T) {
     using C = BwdCfg<MODE, DP>;
     constexpr int BC = C::BC, KS = C::KS, NPAIR = C::NPAIR;
-    constexpr int SLICES = BC / 16;     // 16-column slices per tile = k-steps of the output GEMMs
-    constexpr int GROUPS = 4 / SLICES;  // warp groups that alternate over the tiles
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
     const int q = w & 3, slot = w >> 2;
-    const int sl = slot % SLICES, grp = slot / SLICES;
+    const int sl = slot;  // 16-column slice of every tile = one k-step of the output GEMMs
     const int row = q * 32 + lane;  // owner row inside the CTA tile
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const bool row_valid = row0 + row < p.N;
@@ -180,9 +185,9 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         r_cv = p.cvec[grow];
     }
     bool ok = true;
-    for (int j = grp; j < T; j += GROUPS) {
-        const int b = j & 1;
-        if (!ptx::mbar_wait(bar(C::B_SFULL + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+    for (int j = 0; j < T; ++j) {
+        const int b = NPAIR == 1 ? (j & 1) : 0, sph = NPAIR == 1 ? (j >> 1) & 1 : (j & 1);
+        if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
         const float* st = stats + (j % BWD_STATS_STAGES) * 4 * 64 + 16 * sl;
         if (C::TRANSPOSED)
             if (!ptx::mbar_wait(bar(C::B_STFULL + j % BWD_STATS_STAGES), (j / BWD_STATS_STAGES) & 1, abort_flag,
@@ -216,50 +221,61 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             ptx::tmem_st8(sbase, pa0);
             ptx::tmem_st8(sbase + BC, pa1);
         } else {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t s1[8], s2[8], s3[8], s4[8];
-                ptx::tmem_ld8(sbase + 8 * h, s1);
-                ptx::tmem_ld8(sbase + BC + 8 * h, s2);
-                ptx::tmem_ld8(sbase + 2 * BC + 8 * h, s3);
-                ptx::tmem_ld8(sbase + 3 * BC + 8 * h, s4);
+            // ---- phase A: P and Nn from (S, Sd); then that half of the buffer may be overwritten
+            float P[16], Nn[16], sgv[16], cvv[16];
+            {
+                uint32_t s1[16], s2[16];
+                ptx::tmem_ld16(sbase, s1);
+                ptx::tmem_ld16(sbase + BC, s2);
                 ptx::tmem_wait_ld();
-                uint32_t pa0[4], pa1[4];
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + 1));
 #pragma unroll
-                for (int c4 = 0; c4 < 8; c4 += 4) {
-                    float lv[4], mv[4], gv[4], cvv[4];
+                for (int c4 = 0; c4 < 16; c4 += 4) {
+                    float lv[4], mv[4];
                     if (C::TRANSPOSED) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(st + 8 * h + c4);
-                        const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + 8 * h + c4);
-                        const float4 g4 = *reinterpret_cast<const float4*>(st + 128 + 8 * h + c4);
-                        const float4 c44 = *reinterpret_cast<const float4*>(st + 192 + 8 * h + c4);
+                        const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
+                        const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
+                        const float4 g4 = *reinterpret_cast<const float4*>(st + 128 + c4);
+                        const float4 c44 = *reinterpret_cast<const float4*>(st + 192 + c4);
                         lv[0] = l4.x; lv[1] = l4.y; lv[2] = l4.z; lv[3] = l4.w;
                         mv[0] = m4.x; mv[1] = m4.y; mv[2] = m4.z; mv[3] = m4.w;
-                        gv[0] = g4.x; gv[1] = g4.y; gv[2] = g4.z; gv[3] = g4.w;
-                        cvv[0] = c44.x; cvv[1] = c44.y; cvv[2] = c44.z; cvv[3] = c44.w;
+                        sgv[c4] = g4.x; sgv[c4 + 1] = g4.y; sgv[c4 + 2] = g4.z; sgv[c4 + 3] = g4.w;
+                        cvv[c4] = c44.x; cvv[c4 + 1] = c44.y; cvv[c4 + 2] = c44.z; cvv[c4 + 3] = c44.w;
                     } else {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            lv[e] = (key0 + 8 * h + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
-                            mv[e] = r_mu; gv[e] = r_s1; cvv[e] = r_cv;
+                            lv[e] = (key0 + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
+                            mv[e] = r_mu; sgv[c4 + e] = r_s1; cvv[c4 + e] = r_cv;
                         }
                     }
-                    float a0[4], a1[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        bwd_element<MODE>(p, __uint_as_float(s1[c4 + e]), __uint_as_float(s2[c4 + e]),
-                                          __uint_as_float(s3[c4 + e]), __uint_as_float(s4[c4 + e]), lv[e], mv[e], gv[e],
-                                          cvv[e], a0[e], a1[e]);
-                    pa0[c4 >> 1] = ptx::pack_bf16(a0[0], a0[1]);
-                    pa0[(c4 >> 1) + 1] = ptx::pack_bf16(a0[2], a0[3]);
-                    pa1[c4 >> 1] = ptx::pack_bf16(a1[0], a1[1]);
-                    pa1[(c4 >> 1) + 1] = ptx::pack_bf16(a1[2], a1[3]);
+                    for (int e = 0; e < 4; ++e) {
+                        P[c4 + e] = ptx::ex2(fmaf(__uint_as_float(s1[c4 + e]), p.c2, -lv[e]));
+                        Nn[c4 + e] = fmaf(p.alpha, __uint_as_float(s2[c4 + e]), -mv[e]);
+                    }
                 }
-                // half h of the k-step's operand: 4 packed columns.  They overwrite accumulator columns of
-                // this warp's own slice that it has already read.
-                ptx::tmem_st4(sbase + 4 * h, pa0);
-                ptx::tmem_st4(sbase + BC + 4 * h, pa1);
             }
+            // ---- phase B: W = P (D - Sigma1), dA = P (X - c) + W Nn, written over this slice's D and X columns
+            if (!ptx::mbar_wait(bar(C::B_SFULL + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            uint32_t s3[16], s4[16];
+            ptx::tmem_ld16(sbase + 2 * BC, s3);
+            ptx::tmem_ld16(sbase + 3 * BC, s4);
+            ptx::tmem_wait_ld();
+            uint32_t pa0[8], pa1[8];
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) {
+                const float w0 = P[c] * (__uint_as_float(s3[c]) - sgv[c]);
+                const float w1 = P[c + 1] * (__uint_as_float(s3[c + 1]) - sgv[c + 1]);
+                const float d0 = fmaf(P[c], __uint_as_float(s4[c]) - cvv[c], w0 * Nn[c]);
+                const float d1 = fmaf(P[c + 1], __uint_as_float(s4[c + 1]) - cvv[c + 1], w1 * Nn[c + 1]);
+                pa0[c >> 1] = ptx::pack_bf16(w0, w1);
+                pa1[c >> 1] = ptx::pack_bf16(d0, d1);
+            }
+            ptx::tmem_st8(sbase + 2 * BC, pa0);
+            ptx::tmem_st8(sbase + 3 * BC, pa1);
         }
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
@@ -312,7 +328,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t own_base = ptx::smem_u32(smem);
     const uint32_t e_base = own_base + C::NOWN_SMEM * C::OWN_BYTES;
-    const uint32_t l_base = e_base + SE * 2 * C::ST_BYTES;
+    const uint32_t l_base = e_base + SE * 2 * C::EST_BYTES;
     uint8_t* misc = smem + C::TILE_BYTES;
     const uint32_t bar0 = ptx::smem_u32(misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48 * 8);
@@ -348,14 +364,18 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         // (it pads d to a multiple of 16) and is never written again.  Logical chunk k of row r sits at
         // physical chunk k ^ (r & 7).
         if (((p.d - 64) >> 3) < 2) {
-            for (int i = threadIdx.x; i < C::NOWN_SMEM * BWD_ROWS; i += BWD_THREADS) {
+            for (int i = threadIdx.x; i < C::NOWN_SMEM * BWD_ROWS; i += BWD_THREADS) {  // owners: second chunk block
                 const int t = i / BWD_ROWS, r = i - t * BWD_ROWS;
-                uint8_t* atom2 = smem + t * C::OWN_BYTES + BWD_ROWS * 128;
-                *reinterpret_cast<uint4*>(atom2 + r * 128 + ((1 ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(smem + t * C::OWN_BYTES + BWD_ROWS * 128 + BWD_ROWS * 16 + r * 16) = make_uint4(0, 0, 0, 0);
             }
-            for (int i = threadIdx.x; i < (SE + SL) * 2 * BC; i += BWD_THREADS) {
+            for (int i = threadIdx.x; i < SE * 2 * BC; i += BWD_THREADS) {  // E ring: second chunk block
                 const int t = i / BC, r = i - t * BC;
-                uint8_t* atom2 = smem + C::NOWN_SMEM * C::OWN_BYTES + t * C::ST_BYTES + BC * 128;
+                *reinterpret_cast<uint4*>(smem + C::NOWN_SMEM * C::OWN_BYTES + t * C::EST_BYTES + BC * 128 + BC * 16 + r * 16) =
+                    make_uint4(0, 0, 0, 0);
+            }
+            for (int i = threadIdx.x; i < SL * 2 * BC; i += BWD_THREADS) {  // L ring: chunk 1 of the second swizzle atom
+                const int t = i / BC, r = i - t * BC;
+                uint8_t* atom2 = smem + C::NOWN_SMEM * C::OWN_BYTES + SE * 2 * C::EST_BYTES + t * C::LST_BYTES + BC * 128;
                 *reinterpret_cast<uint4*>(atom2 + r * 128 + ((1 ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
             }
             ptx::fence_proxy_async_smem();
@@ -373,7 +393,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
 
     // shared-memory address of tile j of streamed tensor t (0, 1: E ring; 2, 3: L ring)
     auto tile_addr = [&](int t, int j) -> uint32_t {
-        return t < 2 ? e_base + ((j % SE) * 2 + t) * C::ST_BYTES : l_base + ((j % SL) * 2 + (t - 2)) * C::ST_BYTES;
+        return t < 2 ? e_base + ((j % SE) * 2 + t) * C::EST_BYTES : l_base + ((j % SL) * 2 + (t - 2)) * C::LST_BYTES;
     };
 
     if (warp == 0 || warp == 2) {
@@ -399,7 +419,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     const int r = rem / ntail, k = rem - r * ntail;
                     const bool v = row0 + r < p.N;
                     const __nv_bfloat16* src = p.own[2 + t] + ((size_t)bh * p.N + (v ? row0 + r : 0)) * p.d + 64 + 8 * k;
-                    ptx::cp_async_16(own_base + t * C::OWN_BYTES + BWD_ROWS * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+                    ptx::cp_async_16(own_base + t * C::OWN_BYTES + BWD_ROWS * 128 + k * BWD_ROWS * 16 + r * 16, src, v ? 16u : 0u);
                 }
                 ptx::cp_async_commit();
                 ptx::cp_async_wait<0>();
@@ -409,8 +429,20 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
         }
         bool ok = true;
+        int pending = -1;  // tile whose copied columns have not been signalled yet
         for (int j = 0; j < T; ++j) {
             const int s = j % S, ph = (j / S) & 1;
+            if constexpr (NA == 2) {
+                // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
+                // that tile before it frees the stage.
+                if (pending >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
+                    ptx::cp_async_wait<0>();
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(b_full + pending % S));
+                    pending = -1;
+                }
+            }
             ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
             if (!ok) break;
             if (lane == 0) {
@@ -424,24 +456,27 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     const int grow = j * BC + r;
                     const bool v = grow < p.N;
                     const __nv_bfloat16* src = srcs[t] + ((size_t)bh * p.N + (v ? grow : 0)) * p.d + 64 + 8 * k;
-                    ptx::cp_async_16(tile_addr(2 * ring + t, j) + BC * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+                    const uint32_t tail = tile_addr(2 * ring + t, j) + BC * 128;
+                    ptx::cp_async_16(ring == 0 ? tail + k * BC * 16 + r * 16 : tail + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
                 }
                 ptx::cp_async_commit();
-                if (j > 0) {
+                if (pending >= 0) {  // the tile before: its copies have had a whole iteration to land
                     ptx::cp_async_wait<1>();
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(b_full + (j - 1) % S));
+                    if (lane == 0) ptx::mbar_arrive(bar(b_full + pending % S));
                 }
+                pending = j;
             }
         }
-        if (NA == 2 && ok) {
-            ptx::cp_async_wait<0>();
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(b_full + (T - 1) % S));
+        if (NA == 2) {
+            ptx::cp_async_wait<0>();  // nothing of ours stays in flight
+            if (ok && pending >= 0) {
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(b_full + pending % S));
+            }
         }
-        if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer: the whole warp runs
         // the loop in converged control flow; one elected lane issues (see mma_ts_elect)
@@ -450,69 +485,53 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
         const uint32_t ax0 = tb + C::COL_X0, ax1 = tb + C::COL_X1;
         // owner tiles in shared memory (second score pair), K-major A operands
-        const uint64_t o2d = ptx::smem_desc_sw128(own_base, 16, 1024);
-        const uint64_t o3d = ptx::smem_desc_sw128(own_base + C::OWN_BYTES, 16, 1024);
-        auto issue_scores = [&](int j) -> bool {
+        // K-major descriptor of k-step kk of an E-ring tile / of a shared-memory owner tensor: k-steps 0..3 lie
+        // in the 128-byte-swizzled atom, k-step 4 in the unswizzled block behind it
+        auto e_kdesc = [&](uint32_t tile, int kk) -> uint64_t {
+            return kk < 4 ? ptx::smem_desc_sw128(tile, 16, 1024) + (uint64_t)((kk * 32) >> 4)
+                          : ptx::smem_desc_nosw(tile + BC * 128, BC * 16, 128);
+        };
+        auto own_kdesc = [&](int t, int kk) -> uint64_t {
+            const uint32_t base = own_base + t * C::OWN_BYTES;
+            return kk < 4 ? ptx::smem_desc_sw128(base, 16, 1024) + (uint64_t)((kk * 32) >> 4)
+                          : ptx::smem_desc_nosw(base + BWD_ROWS * 128, BWD_ROWS * 16, 128);
+        };
+        // `ready`: the caller has already seen every barrier of this step complete (mbar_test3_warp)
+        auto issue_scores = [&](int j, bool ready) -> bool {
             const int b = j & 1;
-            if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-            if (NPAIR == 2)
-                if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (!ready) {
+                if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+                if (NPAIR == 2)
+                    if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            }
             ptx::tc_fence_after_sync();
             if (lane == 0) BTL_STAMP(0, j, 0);
-            // first-pair stream operands Y0, Y1: E ring for DV, L ring for DK/DQ; K-major B
-            const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(NPAIR == 1 ? 0 : 2, j), 16, 1024);
-            const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(NPAIR == 1 ? 1 : 3, j), 16, 1024);
+            // DV only (the two-pair passes use the split-phase loop below): Y0, Y1 in the E ring, K-major B
+            const uint32_t t0 = tile_addr(0, j), t1 = tile_addr(1, j);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {  // S = X0 Y0^T
-                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                ptx::mma_ts_elect(dS, ax0 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
-            }
+            for (int kk = 0; kk < KS; ++kk)  // S = X0 Y0^T
+                ptx::mma_ts_elect(dS, ax0 + 8 * kk, e_kdesc(t0, kk), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {  // Sd = X1 Y0^T
-                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                ptx::mma_ts_elect(dT, ax1 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
-            }
+            for (int kk = 0; kk < KS; ++kk)  // Sd = X1 Y0^T
+                ptx::mma_ts_elect(dT, ax1 + 8 * kk, e_kdesc(t0, kk), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {  // Sd += X0 Y1^T
-                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                ptx::mma_ts_elect(dT, ax0 + 8 * kk, y1 + off, idesc_s, 1u);
-            }
-            if (NPAIR == 2) {
-                const uint64_t y2 = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
-                const uint64_t y3 = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
-                const uint32_t dD = dS + 2 * BC, dX = dS + 3 * BC;
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {  // D = X2 Y2^T
-                    const uint64_t offa = (uint64_t)(((kk >> 2) * BWD_ROWS * 128 + (kk & 3) * 32) >> 4);
-                    const uint64_t offb = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ss_elect(dD, o2d + offa, y2 + offb, idesc_s, kk > 0 ? 1u : 0u);
-                }
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {  // X = X3 Y2^T
-                    const uint64_t offa = (uint64_t)(((kk >> 2) * BWD_ROWS * 128 + (kk & 3) * 32) >> 4);
-                    const uint64_t offb = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ss_elect(dX, o3d + offa, y2 + offb, idesc_s, kk > 0 ? 1u : 0u);
-                }
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {  // X += X2 Y3^T
-                    const uint64_t offa = (uint64_t)(((kk >> 2) * BWD_ROWS * 128 + (kk & 3) * 32) >> 4);
-                    const uint64_t offb = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ss_elect(dX, o2d + offa, y3 + offb, idesc_s, 1u);
-                }
-            }
+            for (int kk = 0; kk < KS; ++kk)  // Sd += X0 Y1^T
+                ptx::mma_ts_elect(dT, ax0 + 8 * kk, e_kdesc(t1, kk), idesc_s, 1u);
             ptx::mma_commit_elect(bar(C::B_SFULL + b));
             ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
             if (lane == 0) BTL_STAMP(0, j, 1);
             return true;
         };
-        auto issue_outputs = [&](int j) -> bool {
+        auto issue_outputs = [&](int j, bool ready) -> bool {
             const int b = j & 1;
-            if (NPAIR == 1)
-                if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             if (lane == 0) BTL_STAMP(0, j, 2);
-            if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-            ptx::tc_fence_after_sync();
+            if (!ready) {
+                if (NPAIR == 1)
+                    if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+                if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+                ptx::tc_fence_after_sync();
+            }
             if (lane == 0) BTL_STAMP(0, j, 3);
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B (the L ring): atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
@@ -535,10 +554,103 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, BWD_WAIT_LIMIT_NS);
         if (ok && NPAIR == 2) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), 0, abort_flag, BWD_WAIT_LIMIT_NS);
         ptx::tc_fence_after_sync();
-        if (ok) ok = issue_scores(0);
-        for (int j = 0; ok && j < T; ++j) {
-            if (j + 1 < T) ok = issue_scores(j + 1);
-            if (ok) ok = issue_outputs(j);
+        if constexpr (NPAIR == 1) {
+            if (ok) ok = issue_scores(0, false);
+            for (int j = 0; ok && j < T; ++j) {
+                // one combined poll of what the two steps below wait for
+                bool ready = false;
+                if (j + 1 < T) {
+                    const int jn = j + 1;
+                    ready = ptx::mbar_test3_warp(bar(C::B_EFULL + jn % SE), (jn / SE) & 1, bar(C::B_LFULL + j % SL), (j / SL) & 1,
+                                                 bar(C::B_PREADY + (j & 1)), (j >> 1) & 1);
+                    ok = issue_scores(jn, ready);
+                }
+                if (ok) ok = issue_outputs(j, ready);
+            }
+        } else {
+            // One score buffer used in two phases.  Order on the tensor pipe:
+            //   (S, Sd)(0), (D, X)(0), then per tile j: (S, Sd)(j+1) once the element-wise warps have read
+            //   (S, Sd)(j) | outputs(j) once the operands W, dA are written | (D, X)(j+1), which overwrites them.
+            const uint32_t dS = tb + C::COL_SCORE, dT = dS + BC, dD = dS + 2 * BC, dX = dS + 3 * BC;
+            auto issue_first_pair = [&](int j) {  // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; Y0, Y1 in the L ring, K-major
+                const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, j), 16, 1024);
+                const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, j), 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dS, ax0 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dT, ax1 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dT, ax0 + 8 * kk, y1 + off, idesc_s, 1u);
+                }
+                ptx::mma_commit_elect(bar(C::B_SFULL + 0));
+            };
+            auto issue_second_pair = [&](int j) {  // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; Y2, Y3 in the E ring
+                const uint32_t t2 = tile_addr(0, j), t3 = tile_addr(1, j);
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dD, own_kdesc(0, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(1, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+#pragma unroll
+                for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(0, kk), e_kdesc(t3, kk), idesc_s, 1u);
+                ptx::mma_commit_elect(bar(C::B_SFULL + 1));
+                ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+            };
+            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                issue_first_pair(0);
+                issue_second_pair(0);
+            }
+            for (int j = 0; ok && j < T; ++j) {
+                if (j + 1 < T) {
+                    const int jn = j + 1;
+                    // (S, Sd)(j) read by all element-wise warps, and the tiles of j+1 loaded
+                    const bool ready = ptx::mbar_test3_warp(bar(C::B_PREADY + 1), j & 1, bar(C::B_LFULL + jn % SL), (jn / SL) & 1,
+                                                            bar(C::B_EFULL + jn % SE), (jn / SE) & 1);
+                    if (!ready) {
+                        ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + jn % SL), (jn / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + jn % SE), (jn / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    if (lane == 0) BTL_STAMP(0, jn, 0);
+                    issue_first_pair(jn);
+                    if (lane == 0) BTL_STAMP(0, jn, 1);
+                }
+                // outputs(j): acc0 += W B0, acc1 += dA B0 + W B1 with the operands in the D and X columns
+                if (lane == 0) BTL_STAMP(0, j, 2);
+                ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                if (lane == 0) BTL_STAMP(0, j, 3);
+                {
+                    const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);  // MN-major B
+                    const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+                    const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+#pragma unroll
+                    for (int u = 0; u < BC / 16; ++u) {
+                        const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                        const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                        ptx::mma_ts_elect(acc0, dD + 16 * u, b0 + off, idesc_o, acc);
+                        ptx::mma_ts_elect(acc1, dX + 16 * u, b0 + off, idesc_o, acc);
+                        ptx::mma_ts_elect(acc1, dD + 16 * u, b1 + off, idesc_o, 1u);
+                    }
+                    ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+                    if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                }
+                if (lane == 0) BTL_STAMP(0, j, 4);
+                if (j + 1 < T) issue_second_pair(j + 1);
+            }
         }
     } else if (warp == 3) {
         // ------------------------------------------------------------------ per-query statistics (transposed passes):
@@ -548,16 +660,19 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const size_t srow = (size_t)bh * p.N;
             const float* src_stat[4] = {p.lse2, p.mu, p.sig1, p.cvec};
             if ((p.N & 3) == 0) {
-                constexpr int CPS = BC / 4;  // 16-byte chunks per statistic and tile; 32 chunks per tile in all
-                const int stat = lane / CPS, chunk = lane - stat * CPS;
-                const float* src = src_stat[stat] + srow + 4 * chunk;
+                constexpr int CPS = BC / 4;  // 16-byte chunks per statistic and tile
                 bool ok = true;
                 for (int j = 0; j < T; ++j) {
                     const int s = j % BWD_STATS_STAGES, ph = (j / BWD_STATS_STAGES) & 1;
                     ok = ptx::mbar_wait_warp(bar(C::B_STEMPTY + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     if (!ok) break;
-                    const bool v = j * BC + 4 * chunk < p.N;  // queries beyond N read as zero: their B rows are zero too
-                    ptx::cp_async_16(ptx::smem_u32(stats + s * 4 * 64 + stat * 64 + 4 * chunk), src + (v ? j * BC : 0), v ? 16u : 0u);
+#pragma unroll
+                    for (int i = lane; i < 2 * NPAIR * CPS; i += 32) {
+                        const int stat = i / CPS, chunk = i - stat * CPS;
+                        const bool v = j * BC + 4 * chunk < p.N;  // queries beyond N read as zero: their B rows are zero too
+                        ptx::cp_async_16(ptx::smem_u32(stats + s * 4 * 64 + stat * 64 + 4 * chunk),
+                                         src_stat[stat] + srow + (v ? j * BC + 4 * chunk : 0), v ? 16u : 0u);
+                    }
                     ptx::cp_async_commit();
                     if (j >= BWD_STATS_LAG) {
                         ptx::cp_async_wait<BWD_STATS_LAG>();

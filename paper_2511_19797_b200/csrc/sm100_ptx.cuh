@@ -174,6 +174,17 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
     d |= static_cast<uint64_t>(2) << 61;
     return d;
 }
+// Same descriptor without swizzle: core matrices of 8 rows x 16 bytes, each contiguous (128 bytes).
+// For a K-major operand lbo_bytes is the distance between the core matrices of the two 16-byte
+// halves of a k-step, sbo_bytes the distance between 8-row groups.
+__device__ __forceinline__ uint64_t smem_desc_nosw(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    return d;
+}
 // 32-bit instruction descriptor: fp32 accumulate (bits 4-5 = 1), bf16 A and B (bits 7-9, 10-12 = 1),
 // A/B major-ness (bits 15, 16; 0 = K-major, 1 = MN-major), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
 __host__ __device__ constexpr uint32_t idesc_bf16_f32(uint32_t M, uint32_t N, uint32_t a_mn_major, uint32_t b_mn_major) {
@@ -237,6 +248,37 @@ __device__ __forceinline__ void mma_commit_elect(uint32_t bar) {
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
     const bool ok = mbar_wait(bar, parity, abort_flag, limit_ns);
     return __all_sync(0xffffffffu, ok);
+}
+
+// Non-blocking test of one mbarrier phase; warp-uniform result.
+__device__ __forceinline__ bool mbar_test_warp(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return __all_sync(0xffffffffu, ok != 0);
+}
+
+// Non-blocking test of three mbarrier phases at once; the three polls are issued back to back so
+// that their shared-memory round trips overlap.  Warp-uniform result.  In the steady state of a
+// pipeline all three have completed and one round trip replaces three serial waits.
+__device__ __forceinline__ bool mbar_test3_warp(uint32_t b0, uint32_t p0, uint32_t b1, uint32_t p1, uint32_t b2, uint32_t p2) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred a;\n\t.reg .pred b;\n\t.reg .pred c;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 a, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 b, [%3], %4;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 c, [%5], %6;\n\t"
+        "and.pred a, a, b;\n\tand.pred a, a, c;\n\t"
+        "selp.u32 %0, 1, 0, a;\n\t}"
+        : "=r"(ok)
+        : "r"(b0), "r"(p0), "r"(b1), "r"(p1), "r"(b2), "r"(p2)
+        : "memory");
+    return __all_sync(0xffffffffu, ok != 0);
 }
 
 // ---------------------------------------------------------------- small math helpers
