@@ -34,7 +34,8 @@ typedef enum {
     TVM_ATTN_UNSUPPORTED = -2,         /* d > 128 or d % 8 != 0, device is not sm_100, too many tiles  */
     TVM_ATTN_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < tvm_attn_jvp_workspace_bytes(...) */
     TVM_ATTN_CUDA_ERROR = -4,          /* a CUDA runtime/driver call or a launch failed */
-    TVM_ATTN_DEVICE_TIMEOUT = -5       /* a bounded on-device wait ran out (see tvm_attn_check_status) */
+    TVM_ATTN_DEVICE_TIMEOUT = -5,      /* a bounded on-device wait ran out (see tvm_attn_check_status) */
+    TVM_ATTN_TOO_LARGE = -6            /* B*H*N exceeds the built-in scratch of tvm_attn_jvp_bwd_noalloc */
 } tvm_attn_status;
 
 /* dtype of the eight/sixteen (B,H,N,d) tensors */
@@ -97,6 +98,34 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
                      const float* lse, const float* mu, const void* dO, const void* dtO, void* dQ,
                      void* dK, void* dV, void* dtQ, void* dtK, void* dtV, void* workspace,
                      size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward pass for callers that cannot allocate device memory (no counterpart in the paper).
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they need the backward: code
+ * running inside another framework's memory plan with every byte already assigned, a real-time or
+ * embedded loop where an allocation could fail or stall, a plug-in that is handed tensors but no
+ * allocator.  tvm_attn_jvp_bwd asks them for a workspace they have no way to provide.  This entry
+ * point computes exactly what tvm_attn_jvp_bwd computes, with the same arguments minus the workspace,
+ * and keeps its scratch in a fixed array inside the library's device image instead.
+ *
+ *   - Limit: B * H * N <= TVM_ATTN_NOALLOC_MAX_ROWS.  Larger problems return TVM_ATTN_TOO_LARGE before
+ *     anything is launched; use tvm_attn_jvp_bwd with your own workspace for those.
+ *   - Cost: the array (12 bytes per row, 3 MiB) is part of the library image, so every GPU that loads the
+ *     library holds it until the process exits, whether or not this function is ever called.
+ *   - It calls neither cudaMalloc nor cudaFree nor any allocating library routine.
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (the pass rewrites
+ *     all of it before reading it) and its contents after a call are unspecified.  Two calls that may
+ *     run at the same time on the GPU (different streams, different host threads) race on it: serialise
+ *     them, or give the concurrent ones their own workspace through tvm_attn_jvp_bwd.
+ */
+#define TVM_ATTN_NOALLOC_MAX_ROWS 262144
+int tvm_attn_jvp_bwd_noalloc(const tvm_attn_params* p, const void* Q, const void* K, const void* V,
+                             const void* tQ, const void* tK, const void* tV, const void* O, const void* tO,
+                             const float* lse, const float* mu, const void* dO, const void* dtO, void* dQ,
+                             void* dK, void* dV, void* dtQ, void* dtK, void* dtV, void* cuda_stream);
 
 /*
  * Synchronises `cuda_stream` and reports what the kernels enqueued so far on the current device

@@ -16,7 +16,8 @@ FP32 = 1
 FLAG_CUDA_CORES = 1
 
 _STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
-                 -5: "DEVICE_TIMEOUT"}
+                 -5: "DEVICE_TIMEOUT", -6: "TOO_LARGE"}
+NOALLOC_MAX_ROWS = 262144
 
 
 class TvmAttnError(RuntimeError):
@@ -31,7 +32,8 @@ class Params(ctypes.Structure):
 
 
 _lib = None
-EXPORTS = ("tvm_attn_jvp_workspace_bytes", "tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_check_status",
+EXPORTS = ("tvm_attn_jvp_workspace_bytes", "tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_jvp_bwd_noalloc",
+           "tvm_attn_check_status",
            "tvm_attn_launch_count", "tvm_attn_strerror", "tvm_attn_version", "tvm_attn_set_profiling",
            "tvm_attn_get_profile")
 
@@ -59,6 +61,8 @@ def load(build_if_missing=False):
     lib.tvm_attn_jvp_fwd.argtypes = [pp] + [vp] * 10 + [vp, ctypes.c_size_t, vp]
     lib.tvm_attn_jvp_bwd.restype = ctypes.c_int
     lib.tvm_attn_jvp_bwd.argtypes = [pp] + [vp] * 18 + [vp, ctypes.c_size_t, vp]
+    lib.tvm_attn_jvp_bwd_noalloc.restype = ctypes.c_int
+    lib.tvm_attn_jvp_bwd_noalloc.argtypes = [pp] + [vp] * 18 + [vp]
     lib.tvm_attn_check_status.restype = ctypes.c_int
     lib.tvm_attn_check_status.argtypes = [vp]
     lib.tvm_attn_launch_count.restype = ctypes.c_uint64
@@ -149,6 +153,25 @@ def tvm_attn_jvp_bwd(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, scale=0.0, fl
     if rc != 0:
         _raise("tvm_attn_jvp_bwd", rc)
     return outs
+
+
+def tvm_attn_jvp_bwd_noalloc(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, out, scale=0.0, flags=0, stream=None):
+    """Backward for callers that cannot allocate: same result as tvm_attn_jvp_bwd, scratch inside the library.
+
+    `out` must hold the six preallocated gradient tensors (dQ, dK, dV, dtQ, dtK, dtV): this wrapper, like the
+    C entry point behind it, allocates nothing.  B*H*N may not exceed NOALLOC_MAX_ROWS.  Calls that may overlap
+    on the GPU race on the shared scratch; the first call on a device should come before any stream capture."""
+    lib = load()
+    _check_tensors(Q, (K, V, tQ, tK, tV, O, tO, dO, dtO) + tuple(out))
+    p = _params(Q, scale, flags)
+    with torch.cuda.device(Q.device):
+        rc = lib.tvm_attn_jvp_bwd_noalloc(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
+                                          tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
+                                          mu.data_ptr(), dO.data_ptr(), dtO.data_ptr(), *[o.data_ptr() for o in out],
+                                          _stream_ptr(stream))
+    if rc != 0:
+        _raise("tvm_attn_jvp_bwd_noalloc", rc)
+    return tuple(out)
 
 
 def tvm_attn_check_status(stream=None, raise_on_error=True):

@@ -277,6 +277,28 @@ static TcParams base_params(const Shape& s, int* status) {
     return prm;
 }
 
+// Scratch of tvm_attn_jvp_bwd_noalloc: three floats per row, for callers that cannot allocate.  In host code
+// this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) float g_noalloc_scratch[3 * TVM_ATTN_NOALLOC_MAX_ROWS];
+static constexpr int kMaxDevices = 64;
+static float* g_noalloc_addr[kMaxDevices] = {};  // device address of the array, per device
+static std::mutex g_noalloc_mutex;
+
+// Device address of the scratch array on the current device, looked up on first use.
+static int noalloc_scratch_address(float** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TVM_ATTN_CUDA_ERROR;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_addr[dev]) {
+        float* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch) != cudaSuccess || !ptr)
+            return TVM_ATTN_CUDA_ERROR;
+        g_noalloc_addr[dev] = ptr;
+    }
+    *out = g_noalloc_addr[dev];
+    return TVM_ATTN_OK;
+}
+
 }  // namespace tvm_attn
 
 using namespace tvm_attn;
@@ -433,6 +455,21 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     return rc;
 }
 
+int tvm_attn_jvp_bwd_noalloc(const tvm_attn_params* p, const void* Q, const void* K, const void* V, const void* tQ,
+                             const void* tK, const void* tV, const void* O, const void* tO, const float* lse,
+                             const float* mu, const void* dO, const void* dtO, void* dQ, void* dK, void* dV, void* dtQ,
+                             void* dtK, void* dtV, void* cuda_stream) {
+    Shape s;
+    const int rc = check_params(p, &s);
+    if (rc != TVM_ATTN_OK) return rc;
+    if (s.BH * (long long)s.N > (long long)TVM_ATTN_NOALLOC_MAX_ROWS) return TVM_ATTN_TOO_LARGE;
+    float* scratch = nullptr;
+    const int rs = noalloc_scratch_address(&scratch);
+    if (rs != TVM_ATTN_OK) return rs;
+    return tvm_attn_jvp_bwd(p, Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, dQ, dK, dV, dtQ, dtK, dtV, scratch,
+                            sizeof(float) * 3 * (size_t)TVM_ATTN_NOALLOC_MAX_ROWS, cuda_stream);
+}
+
 int tvm_attn_check_status(void* cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
     int host = 0;
@@ -471,6 +508,8 @@ const char* tvm_attn_strerror(int code) {
         case TVM_ATTN_WORKSPACE_TOO_SMALL: return "workspace smaller than tvm_attn_jvp_workspace_bytes()";
         case TVM_ATTN_CUDA_ERROR: return "a CUDA call or kernel launch failed";
         case TVM_ATTN_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out; outputs are unspecified";
+        case TVM_ATTN_TOO_LARGE: return "B*H*N exceeds TVM_ATTN_NOALLOC_MAX_ROWS, the built-in scratch of tvm_attn_jvp_bwd_noalloc; "
+                                        "call tvm_attn_jvp_bwd with a workspace instead";
         default: return "unknown status";
     }
 }
