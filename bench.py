@@ -58,7 +58,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
             return
@@ -70,6 +70,16 @@ class ClockSampler:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) >= 7:
                 self.rows.append(parts)
+
+    def wait_first(self, timeout=5.0):
+        """Blocks until nvidia-smi has delivered its first sample (it takes a moment to start)."""
+        t0 = time.time()
+        while self.proc is not None and not self.rows and time.time() - t0 < timeout:
+            time.sleep(0.02)
+
+    def mark(self):
+        """Samples taken before this call are dropped: only the timed region is summarised."""
+        self.rows = []
 
     def stop(self):
         if self.proc is None:
@@ -92,7 +102,7 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_sample(wl_name, target_seconds=12.0, threads=None):
+def oracle_sample(wl_name, target_seconds=12.0, threads=None, heads=None):
     """Times the C oracle (forward + backward) on a bounded sample of whole heads of the workload.
     Returns (TFLOP/s, threads, description, seconds)."""
     import numpy as np
@@ -102,21 +112,37 @@ def oracle_sample(wl_name, target_seconds=12.0, threads=None):
     wl = inputs.WORKLOADS[wl_name]
     cores = threads or c_oracle.default_threads()
     f_fwd, f_bwd = inputs.flops(1, 1, wl.N, wl.d)
-    est_rate = 0.25e9 * 2  # ~FLOP/s of one thread of the plain C loops; only sizes the sample
-    heads = int(max(1, min(wl.B * wl.H, round(target_seconds * est_rate * cores / (f_fwd + f_bwd)))))
-    if heads >= cores:
-        heads = max(cores, heads // cores * cores)
+    alpha = inputs.default_scale(wl.d)
+    if heads is None:
+        heads = calibrate_heads(wl, cores, alpha, target_seconds)
     idx = [int(i) for i in np.linspace(0, wl.B * wl.H - 1, heads).round()]
     x = inputs.make_inputs(wl, heads=idx)
     xs = [x[k].to(torch.bfloat16).to(torch.float64).numpy() for k in inputs.NAMES]
-    alpha = inputs.default_scale(wl.d)
     t0 = time.perf_counter()
     used = c_oracle.attn_jvp_fwd(*xs[:6], alpha, nthreads=cores)[4]
     c_oracle.attn_jvp_bwd(*xs, alpha, nthreads=cores)
     dt = time.perf_counter() - t0
     tflops = heads * (f_fwd + f_bwd) / dt / 1e12
     desc = "%d of %d heads of %s (fwd+bwd, fp64 C oracle, gcc -O2), %.1f s" % (heads, wl.B * wl.H, wl_name, dt)
-    return tflops, used, desc, dt
+    return tflops, used, desc, dt, heads
+
+
+def calibrate_heads(wl, cores, alpha, target_seconds):
+    """Times one head per thread and returns how many whole heads make about `target_seconds` of CPU work."""
+    import torch
+    from oracle import c_oracle
+    from paper_2511_19797_b200 import inputs
+    probe = min(cores, wl.B * wl.H)
+    xp = inputs.make_inputs(wl, heads=list(range(probe)))
+    xps = [xp[k].to(torch.bfloat16).to(torch.float64).numpy() for k in inputs.NAMES]
+    t0 = time.perf_counter()
+    c_oracle.attn_jvp_fwd(*xps[:6], alpha, nthreads=cores)
+    c_oracle.attn_jvp_bwd(*xps, alpha, nthreads=cores)
+    t_probe = max(time.perf_counter() - t0, 1e-3)
+    heads = int(max(1, min(wl.B * wl.H, round(probe * target_seconds / t_probe))))
+    if heads >= cores:
+        heads = max(cores, heads // cores * cores)
+    return heads
 
 
 def run_reference(args, rank):
@@ -125,8 +151,11 @@ def run_reference(args, rank):
     from paper_2511_19797_b200 import inputs
     wl = inputs.WORKLOADS[args.workload]
     times, vals = [], []
+    # each step is a bounded sample; the whole run stays within a few minutes whatever K and W are
+    per_step = max(0.25, min(6.0, 150.0 / max(1, args.warmup + args.steps)))
+    heads = None
     for it in range(args.warmup + args.steps):
-        v, cores, desc, dt = oracle_sample(args.workload, target_seconds=6.0)
+        v, cores, desc, dt, heads = oracle_sample(args.workload, target_seconds=per_step, heads=heads)
         if it >= args.warmup:
             times.append(dt); vals.append(v)
     value = statistics.mean(vals)
@@ -146,7 +175,7 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="dit512")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -225,6 +254,8 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        sampler.wait_first()
+        sampler.mark()
     launches0 = binding.tvm_attn_launch_count()
     ms_total = timed(step, args.steps)
     launches = binding.tvm_attn_launch_count() - launches0
@@ -307,7 +338,7 @@ def main():
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        v, cores, desc, _ = oracle_sample(args.workload)
+        v, cores, desc, _, _ = oracle_sample(args.workload)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
     else:
         line["cpu_baseline"] = None
