@@ -30,6 +30,9 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # GEMMs each kernel executes by design (x 2*B*H*N^2*d FLOP each, true d)
 KERNEL_GEMMS = {"fwd": 6, "bwd_rowsums": 0, "bwd_dv": 6, "bwd_dk": 9, "bwd_dq": 9}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/jvp_fwd_bwd_kernels_dit512.md (that workload only; None for anything else)
+NCU_TRAFFIC_BYTES = {"dit512": {"fwd": 281.7e6, "bwd_dv": 287.9e6, "bwd_dk": 370.0e6, "bwd_dq": 364.7e6}}
 
 
 def load_peaks():
@@ -329,7 +332,8 @@ def main():
         "kernels_share": {k: v / total_k for k, v in kernel_ms.items()},
         "roofline": {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "peak_source": peak_src + " (sustained bf16 GEMM; kernel timed inside a long step)",
-                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "traffic": None,
+                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get(top),
                      "flops_per_launch": KERNEL_GEMMS[top] * unit_flops},
         "e2e": None if ms_e2e is None else {
             "value": world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
