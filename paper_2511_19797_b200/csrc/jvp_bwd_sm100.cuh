@@ -281,6 +281,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);
+        if (lane == 0) BTL_STAMP(4 + (w >> 3), j, w & 7);
         if (lane == 0) {
             ptx::mbar_arrive(bar(C::B_PREADY + b));
             if (C::TRANSPOSED) ptx::mbar_arrive(bar(C::B_STEMPTY + j % BWD_STATS_STAGES));

@@ -81,8 +81,8 @@ struct FwdCfg {
     static constexpr int B_LEMPTY = B_LFULL + SL;
     static constexpr int B_SFULL = B_LEMPTY + SL;
     static constexpr int B_PREADY = B_SFULL + 2;
-    static constexpr int B_OUTDONE = B_PREADY + 2;
-    static constexpr int B_FINAL = B_OUTDONE + 1;
+    static constexpr int B_OUTDONE = B_PREADY + 2;  // per score buffer: the value MMAs that read it have completed
+    static constexpr int B_FINAL = B_OUTDONE + 2;
     static constexpr int B_QREADY = B_FINAL + 1;
     static constexpr int B_XMAX = B_QREADY + 1;   // per quadrant: slice maxima exchanged
     static constexpr int B_XSLOW = B_XMAX + 4;    // per quadrant: slow-path / epilogue exchange
@@ -203,7 +203,7 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             }
             if (j > 0) {
                 // accumulators must be at rest: the value MMAs of tile j-1 have completed
-                if (!ptx::mbar_wait(bar(C::B_OUTDONE), (j - 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                if (!ptx::mbar_wait(bar(C::B_OUTDONE + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
                 for (int ch = sl; ch < KS; ch += 4) {
                     uint32_t o[16], r[16];
@@ -339,6 +339,7 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             ptx::mbar_init(bar(C::B_PREADY + b), 16);
         }
         ptx::mbar_init(bar(C::B_OUTDONE), 1);
+        ptx::mbar_init(bar(C::B_OUTDONE + 1), 1);
         ptx::mbar_init(bar(C::B_FINAL), 1);
         ptx::mbar_init(bar(C::B_QREADY), 16);
         for (int q = 0; q < 4; ++q) { ptx::mbar_init(bar(C::B_XMAX + q), 4); ptx::mbar_init(bar(C::B_XSLOW + q), 4); }
@@ -419,67 +420,68 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        {   // the whole warp runs the loop; one elected lane issues (see mma_ts_elect)
-            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
-            constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
-            const uint32_t aq = tmem_base + C::COL_Q, atq = tmem_base + C::COL_TQ;
-            auto issue_scores = [&](int j) -> bool {
-                const int b = j & 1;
-                if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
-                ptx::tc_fence_after_sync();
-                const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
-                const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
-                const uint32_t dS = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {  // S = Q K^T
-                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ts_elect(dS, aq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
-                }
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {  // Sd = tQ K^T
-                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ts_elect(dT, atq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
-                }
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {  // Sd += Q tK^T
-                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
-                }
-                ptx::mma_commit_elect(bar(C::B_SFULL + b));
-                ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
-                return true;
-            };
-            auto issue_outputs = [&](int j) -> bool {
-                const int b = j & 1;
-                if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
-                if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
-                ptx::tc_fence_after_sync();
-                const uint32_t a0 = tmem_base + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
-                // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
-                const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
-                const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
-                const uint32_t acc0 = tmem_base + C::COL_ACC0, acc1 = tmem_base + C::COL_ACC1;
-#pragma unroll
-                for (int u = 0; u < BC / 16; ++u) {
-                    const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
-                    const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                    ptx::mma_ts_elect(acc0, a0 + 16 * u, vd + off, idesc_o, acc);   // O~ += P~ V
-                    ptx::mma_ts_elect(acc1, a1 + 16 * u, vd + off, idesc_o, acc);   // R  += P~(T-c) V
-                    ptx::mma_ts_elect(acc1, a0 + 16 * u, tvd + off, idesc_o, 1u);   // R  += P~ tV
-                }
-                ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
-                ptx::mma_commit_elect(bar(C::B_OUTDONE));
-                if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
-                return true;
-            };
-            bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, FWD_WAIT_LIMIT_NS);
+        // ------------------------------------------------------------------ score MMAs (warp 1) and value MMAs
+        // (warp 3), on two schedulers: an MMA costs 7 to 14 issue slots of its scheduler, which the element-wise
+        // warps of that quadrant also need.  Each whole warp runs its loop in converged control flow; one
+        // elected lane issues (see mma_ts_elect).
+        constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
+        const uint32_t aq = tb + C::COL_Q, atq = tb + C::COL_TQ;
+        bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, FWD_WAIT_LIMIT_NS);
+        for (int j = 0; ok && j < T; ++j) {
+            const int b = j & 1;
+            ok = ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            // the score buffer is free once the value MMAs of tile j-2 have read their operands out of it
+            if (ok && j >= 2) ok = ptx::mbar_wait_warp(bar(C::B_OUTDONE + b), ((j - 2) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (!ok) break;
             ptx::tc_fence_after_sync();
-            if (ok) ok = issue_scores(0);
-            for (int j = 0; ok && j < T; ++j) {
-                if (j + 1 < T) ok = issue_scores(j + 1);
-                if (ok) ok = issue_outputs(j);
+            const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
+            const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
+            const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {  // S = Q K^T
+                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                ptx::mma_ts_elect(dS, aq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
             }
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {  // Sd = tQ K^T
+                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                ptx::mma_ts_elect(dT, atq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
+            }
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {  // Sd += Q tK^T
+                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
+            }
+            ptx::mma_commit_elect(bar(C::B_SFULL + b));
+            ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+        }
+    } else if (warp == 3) {
+        constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+        bool ok = true;
+        for (int j = 0; ok && j < T; ++j) {
+            const int b = j & 1;
+            ok = ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
+            // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
+            const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
+            const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+#pragma unroll
+            for (int u = 0; u < BC / 16; ++u) {
+                const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                ptx::mma_ts_elect(acc0, a0 + 16 * u, vd + off, idesc_o, acc);   // O~ += P~ V
+                ptx::mma_ts_elect(acc1, a1 + 16 * u, vd + off, idesc_o, acc);   // R  += P~(T-c) V
+                ptx::mma_ts_elect(acc1, a0 + 16 * u, tvd + off, idesc_o, 1u);   // R  += P~ tV
+            }
+            ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+            ptx::mma_commit_elect(bar(C::B_OUTDONE + b));
+            if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
         }
     } else if (warp >= 4) {
         fwd_elementwise<DP>(p, tmem_base, bar0, abort_flag, xmax, xslow, warp - 4, lane, bh, row0, T);

@@ -413,7 +413,7 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         }
         {   // dtK = alpha W^T Q, dK = alpha (dA^T Q + W^T tQ) : owner keys (K, tK, V, tV); stream (Hc, G | Q, tQ)
             BwdParams q = b; q.out_scale = s.alpha;
-            if (q.tl) q.tl += 4 * 64 * 8;
+            if (q.tl) q.tl += 6 * 64 * 8;
             q.out0 = static_cast<__nv_bfloat16*>(dtK); q.out1 = static_cast<__nv_bfloat16*>(dK);
             const void* own[4] = {K, tK, V, tV};
             const void* strm[4] = {dtO, dO, Q, tQ};
@@ -422,7 +422,7 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         }
         {   // dtQ = alpha W K, dQ = alpha (dA K + W tK) : owner queries (Q, tQ, Hc, G); stream (V, tV | K, tK)
             BwdParams q = b; q.out_scale = s.alpha;
-            if (q.tl) q.tl += 2 * 4 * 64 * 8;
+            if (q.tl) q.tl += 2 * 6 * 64 * 8;
             q.out0 = static_cast<__nv_bfloat16*>(dtQ); q.out1 = static_cast<__nv_bfloat16*>(dQ);
             const void* own[4] = {Q, tQ, dtO, dO};
             const void* strm[4] = {V, tV, K, tK};
