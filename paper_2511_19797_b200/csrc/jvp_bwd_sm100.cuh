@@ -221,8 +221,10 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             ptx::tmem_st8(sbase, pa0);
             ptx::tmem_st8(sbase + BC, pa1);
         } else {
-            // ---- phase A: P and Nn from (S, Sd); then that half of the buffer may be overwritten
-            float P[16], Nn[16], sgv[16], cvv[16];
+            // ---- phase A: P, Nn, -P Sigma1, -P c from (S, Sd), two columns per register pair; then that half of the
+            // buffer may be overwritten.  Phase B, which sits on the critical path between the second score pair and
+            // the output MMAs, is left with three packed FMAs per column pair.
+            uint64_t P2[8], Nn2[8], nPs2[8], nPc2[8];
             {
                 uint32_t s1[16], s2[16];
                 ptx::tmem_ld16(sbase, s1);
@@ -231,9 +233,10 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + 1));
+                const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
 #pragma unroll
                 for (int c4 = 0; c4 < 16; c4 += 4) {
-                    float lv[4], mv[4];
+                    float lv[4], mv[4], gv[4], cv[4];
                     if (C::TRANSPOSED) {
                         const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
                         const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
@@ -241,23 +244,29 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                         const float4 c44 = *reinterpret_cast<const float4*>(st + 192 + c4);
                         lv[0] = l4.x; lv[1] = l4.y; lv[2] = l4.z; lv[3] = l4.w;
                         mv[0] = m4.x; mv[1] = m4.y; mv[2] = m4.z; mv[3] = m4.w;
-                        sgv[c4] = g4.x; sgv[c4 + 1] = g4.y; sgv[c4 + 2] = g4.z; sgv[c4 + 3] = g4.w;
-                        cvv[c4] = c44.x; cvv[c4 + 1] = c44.y; cvv[c4 + 2] = c44.z; cvv[c4 + 3] = c44.w;
+                        gv[0] = g4.x; gv[1] = g4.y; gv[2] = g4.z; gv[3] = g4.w;
+                        cv[0] = c44.x; cv[1] = c44.y; cv[2] = c44.z; cv[3] = c44.w;
                     } else {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             lv[e] = (key0 + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
-                            mv[e] = r_mu; sgv[c4 + e] = r_s1; cvv[c4 + e] = r_cv;
+                            mv[e] = r_mu; gv[e] = r_s1; cv[e] = r_cv;
                         }
                     }
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        P[c4 + e] = ptx::ex2(fmaf(__uint_as_float(s1[c4 + e]), p.c2, -lv[e]));
-                        Nn[c4 + e] = fmaf(p.alpha, __uint_as_float(s2[c4 + e]), -mv[e]);
+                    for (int e = 0; e < 4; e += 2) {
+                        const int k = (c4 + e) >> 1;
+                        const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
+                        float x0, x1;
+                        ptx::unpack2(x2, x0, x1);
+                        P2[k] = ptx::pack2(ptx::ex2(x0), ptx::ex2(x1));
+                        Nn2[k] = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
+                        nPs2[k] = ptx::mul2(P2[k], ptx::pack2(-gv[e], -gv[e + 1]));
+                        nPc2[k] = ptx::mul2(P2[k], ptx::pack2(-cv[e], -cv[e + 1]));
                     }
                 }
             }
-            // ---- phase B: W = P (D - Sigma1), dA = P (X - c) + W Nn, written over this slice's D and X columns
+            // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
             if (!ptx::mbar_wait(bar(C::B_SFULL + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             uint32_t s3[16], s4[16];
@@ -266,13 +275,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             ptx::tmem_wait_ld();
             uint32_t pa0[8], pa1[8];
 #pragma unroll
-            for (int c = 0; c < 16; c += 2) {
-                const float w0 = P[c] * (__uint_as_float(s3[c]) - sgv[c]);
-                const float w1 = P[c + 1] * (__uint_as_float(s3[c + 1]) - sgv[c + 1]);
-                const float d0 = fmaf(P[c], __uint_as_float(s4[c]) - cvv[c], w0 * Nn[c]);
-                const float d1 = fmaf(P[c + 1], __uint_as_float(s4[c + 1]) - cvv[c + 1], w1 * Nn[c + 1]);
-                pa0[c >> 1] = ptx::pack_bf16(w0, w1);
-                pa1[c >> 1] = ptx::pack_bf16(d0, d1);
+            for (int k = 0; k < 8; ++k) {
+                const uint64_t w2 = ptx::fma2(P2[k], ptx::pack2u(s3[2 * k], s3[2 * k + 1]), nPs2[k]);
+                const uint64_t t2 = ptx::fma2(P2[k], ptx::pack2u(s4[2 * k], s4[2 * k + 1]), nPc2[k]);
+                const uint64_t d2 = ptx::fma2(w2, Nn2[k], t2);
+                float w0, w1, d0, d1;
+                ptx::unpack2(w2, w0, w1);
+                ptx::unpack2(d2, d0, d1);
+                pa0[k] = ptx::pack_bf16(w0, w1);
+                pa1[k] = ptx::pack_bf16(d0, d1);
             }
             ptx::tmem_st8(sbase + 2 * BC, pa0);
             ptx::tmem_st8(sbase + 3 * BC, pa1);
