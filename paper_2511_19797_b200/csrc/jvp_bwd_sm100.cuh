@@ -202,20 +202,25 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             ptx::tmem_ld16(sbase + BC, s2);
             ptx::tmem_wait_ld();
             uint32_t pa0[8], pa1[8];
+            const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
 #pragma unroll
             for (int c4 = 0; c4 < 16; c4 += 4) {
                 const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
                 const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
                 const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
-                float a0[4], a1[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    bwd_element<MODE>(p, __uint_as_float(s1[c4 + e]), __uint_as_float(s2[c4 + e]), 0.f, 0.f, lv[e], mv[e], 0.f,
-                                      0.f, a0[e], a1[e]);
-                pa0[c4 >> 1] = ptx::pack_bf16(a0[0], a0[1]);
-                pa0[(c4 >> 1) + 1] = ptx::pack_bf16(a0[2], a0[3]);
-                pa1[c4 >> 1] = ptx::pack_bf16(a1[0], a1[1]);
-                pa1[(c4 >> 1) + 1] = ptx::pack_bf16(a1[2], a1[3]);
+                for (int e = 0; e < 4; e += 2) {  // P = 2^(c2 s - lse2), P Nn with Nn = alpha ts - mu: two columns per instruction
+                    const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
+                    float x0, x1;
+                    ptx::unpack2(x2, x0, x1);
+                    const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                    const uint64_t n2 = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
+                    const uint64_t q2 = ptx::mul2(ptx::pack2(p0, p1), n2);
+                    float q0, q1;
+                    ptx::unpack2(q2, q0, q1);
+                    pa0[(c4 + e) >> 1] = ptx::pack_bf16(p0, p1);
+                    pa1[(c4 + e) >> 1] = ptx::pack_bf16(q0, q1);
+                }
             }
             // operand of k-step sl (16 stream rows) sits at column 16*sl of the accumulator it replaces
             ptx::tmem_st8(sbase, pa0);
