@@ -79,8 +79,8 @@ struct FwdCfg {
     static constexpr int B_EEMPTY = B_EFULL + SE;
     static constexpr int B_LFULL = B_EEMPTY + SE;
     static constexpr int B_LEMPTY = B_LFULL + SL;
-    static constexpr int B_SFULL = B_LEMPTY + SL;
-    static constexpr int B_PREADY = B_SFULL + 2;
+    static constexpr int B_SFULL = B_LEMPTY + SL;    // per score buffer: S written (+0, +1), Sd written (+2, +3)
+    static constexpr int B_PREADY = B_SFULL + 4;
     static constexpr int B_OUTDONE = B_PREADY + 2;  // per score buffer: the value MMAs that read it have completed
     static constexpr int B_FINAL = B_OUTDONE + 2;
     static constexpr int B_QREADY = B_FINAL + 1;
@@ -138,12 +138,12 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
 
     for (int j = 0; j < T; ++j) {
         const int b = j & 1;
+        // S is complete before Sd: the row maxima are found and exchanged while the Sd MMAs still run
         if (!ptx::mbar_wait(bar(C::B_SFULL + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS;
         uint32_t s[16], ts[16];
         ptx::tmem_ld16(sbase + 16 * sl, s);
-        ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
         ptx::tmem_wait_ld();
         const int nvalid = p.N - j * BC - 16 * sl;  // columns of this slice that are real keys
         if (nvalid < 16) {
@@ -160,9 +160,13 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
         xm[row * 4 + sl] = mx;
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(bar(C::B_XMAX + q));
+        if (!ptx::mbar_wait(bar(C::B_SFULL + 2 + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
         if (!ptx::mbar_wait(bar(C::B_XMAX + q), j & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         const float4 o4 = *reinterpret_cast<const float4*>(xm + row * 4);
         const float mrow = fmaxf(ptx::max3(o4.x, o4.y, o4.z), o4.w) * p.c2;  // tile maximum of the row, log2 units
+        ptx::tmem_wait_ld();
         const bool need = mrow > m_ref + FWD_LAZY_LOG2;
         if (__any_sync(0xffffffffu, need)) {
             // ---- slow path, taken by the four warps of the quadrant together
@@ -336,6 +340,7 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar(C::B_SFULL + b), 1);
+            ptx::mbar_init(bar(C::B_SFULL + 2 + b), 1);
             ptx::mbar_init(bar(C::B_PREADY + b), 16);
         }
         ptx::mbar_init(bar(C::B_OUTDONE), 1);
@@ -443,6 +448,7 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
                 ptx::mma_ts_elect(dS, aq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
             }
+            ptx::mma_commit_elect(bar(C::B_SFULL + b));
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk) {  // Sd = tQ K^T
                 const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
@@ -453,7 +459,7 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
                 ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
             }
-            ptx::mma_commit_elect(bar(C::B_SFULL + b));
+            ptx::mma_commit_elect(bar(C::B_SFULL + 2 + b));
             ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
         }
     } else if (warp == 3) {
