@@ -314,3 +314,21 @@ def test_tangent_path_matches_the_six_step_equations(bwd):
     got = bwd(Q, K, V, tQ, tK, tV, np.zeros_like(Hc), Hc, alpha)
     for a, b in zip(got, (dQ, dK, dV, dtQ, dtK, dtV)):
         _close(a[0, 0], b, 1e-13)
+
+
+def test_numpy_oracle_accepts_a_subset_of_query_rows():
+    """Queries are independent of one another (App. C Eq. "sdpa": one softmax per query row), so the numpy
+    oracle called with fewer query rows than keys must return exactly those rows of O, tO, lse, mu, dQ, dtQ.
+    The GPU test of the longest sequence relies on this."""
+    xs = _inputs(1, 2, 23, 8, seed=11)
+    rows = [0, 7, 22]
+    sub = lambda a: np.ascontiguousarray(a[:, :, rows])
+    Q, K, V, tQ, tK, tV, G, Hc = xs
+    full_f = onp.attn_jvp_fwd(Q, K, V, tQ, tK, tV, 0.37)
+    part_f = onp.attn_jvp_fwd(sub(Q), K, V, sub(tQ), tK, tV, 0.37)
+    for a, b in zip(part_f, full_f):
+        _close(a, b[:, :, rows], 1e-14)
+    full_b = onp.attn_jvp_bwd(Q, K, V, tQ, tK, tV, G, Hc, 0.37)
+    part_b = onp.attn_jvp_bwd(sub(Q), K, V, sub(tQ), tK, tV, sub(G), sub(Hc), 0.37)
+    _close(part_b[0], full_b[0][:, :, rows], 1e-14)
+    _close(part_b[3], full_b[3][:, :, rows], 1e-14)

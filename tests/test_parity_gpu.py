@@ -48,7 +48,7 @@ def test_full_size_workloads_on_sampled_heads(name, heads):
 
 @pytest.mark.parametrize("B,H,N,d", [
     (1, 1, 1, 8), (1, 2, 7, 16), (2, 1, 64, 64), (1, 1, 100, 72), (1, 3, 129, 40), (2, 2, 191, 128),
-    (1, 1, 257, 72), (1, 2, 320, 32), (1, 1, 1000, 24),
+    (1, 1, 257, 72), (1, 2, 320, 32), (1, 1, 1000, 24), (1, 2, 130, 80), (2, 1, 96, 56), (1, 1, 66, 104),
 ])
 @pytest.mark.parametrize("mode", ["bf16", "fp32"])
 def test_ragged_and_degenerate_shapes(B, H, N, d, mode):
@@ -105,3 +105,36 @@ def test_errors_reported_on_the_gpu_box():
                                  workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.code == -3
     assert binding.tvm_attn_launch_count() >= 0
+
+
+def test_longest_sequence_on_sampled_query_rows():
+    """N = 16384 (the longest sweep point) on a reduced batch: whole heads are too slow for the CPU oracle, but
+    the numpy oracle accepts fewer query rows than keys, so sampled rows of O, tO, lse, mu, dQ and dtQ are
+    compared element by element; the key-side gradients are checked through the identity
+    sum_j dV_j = sum_i (G_i + Hc_i (sum_j Pd_ij)) = sum_i G_i  (rows of P sum to 1, rows of Pd to 0)
+    and sum_j dtV_j = sum_i Hc_i, which hold at any size."""
+    from oracle import attn_jvp_numpy as onp
+    wl = inputs.custom(1, 2, 16384, 64, seed=4, tangent_std=0.5)
+    x = {k: v.to(torch.bfloat16) for k, v in inputs.make_inputs(wl).items()}
+    dev = {k: v.cuda() for k, v in x.items()}
+    O, tO, lse, mu = binding.tvm_attn_jvp_fwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"])
+    grads = binding.tvm_attn_jvp_bwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"], O, tO, lse, mu,
+                                     dev["dO"], dev["dtO"])
+    binding.tvm_attn_check_status()
+    rows = [0, 1, 127, 128, 5000, 8191, 12345, 16383]
+    f64 = {k: v.to(torch.float64).numpy() for k, v in x.items()}
+    sub = lambda k: np.ascontiguousarray(f64[k][:, :, rows])
+    alpha = inputs.default_scale(64)
+    rO, rtO, rlse, rmu = onp.attn_jvp_fwd(sub("Q"), f64["K"], f64["V"], sub("tQ"), f64["tK"], f64["tV"], alpha)
+    rdQ, _, _, rdtQ, _, _ = onp.attn_jvp_bwd(sub("Q"), f64["K"], f64["V"], sub("tQ"), f64["tK"], f64["tV"], sub("dO"),
+                                             sub("dtO"), alpha)
+    pick = lambda t: t.float().cpu().numpy()[:, :, rows]
+    from tests._parity import rel_err
+    errs = {"O": rel_err(pick(O), rO), "tO": rel_err(pick(tO), rtO), "lse": rel_err(pick(lse), rlse),
+            "mu": rel_err(pick(mu), rmu), "dQ": rel_err(pick(grads[0]), rdQ), "dtQ": rel_err(pick(grads[3]), rdtQ)}
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+    dV, dtV = grads[2].double().sum(dim=2).cpu(), grads[5].double().sum(dim=2).cpu()
+    sG, sH = x["dO"].double().sum(dim=2), x["dtO"].double().sum(dim=2)
+    scale = float(sG.abs().max())
+    assert float((dV - sG).abs().max()) <= BF16_BWD * max(scale, 1.0) * 8  # sums of N bf16-rounded rows
+    assert float((dtV - sH).abs().max()) <= BF16_BWD * max(float(sH.abs().max()), 1.0) * 8
