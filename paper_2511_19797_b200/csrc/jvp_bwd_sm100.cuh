@@ -35,6 +35,7 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
+#include <type_traits>
 
 #include "sm100_ptx.cuh"
 
@@ -62,13 +63,16 @@ struct BwdParams {
     const float* sig1;  // rowsum(dtO * O)
     const float* cvec;  // rowsum(dO * O) + rowsum(dtO * tO)
     int* status;        // device status word; non-zero makes the kernel a no-op
-    unsigned long long* tl;  // timeline builds only: clock stamps of CTA 0
+    unsigned long long* tl;  // timeline builds only: clock stamps of one CTA
 };
 
 #ifdef TVM_ATTN_TIMELINE
+#ifndef TVM_ATTN_TIMELINE_CTA
+#define TVM_ATTN_TIMELINE_CTA 0  // the CTA whose clock stamps are recorded
+#endif
 #define BTL_STAMP(role, j, ev)                                                                         \
     do {                                                                                                \
-        if (p.tl && blockIdx.x == 0 && (j) < 64) {                                                      \
+        if (p.tl && blockIdx.x == TVM_ATTN_TIMELINE_CTA && (j) < 64) {                            \
             unsigned long long t_;                                                                      \
             asm volatile("mov.u64 %0, %clock64;" : "=l"(t_));                                          \
             p.tl[((role) * 64 + (j)) * 8 + (ev)] = t_;                                                  \
@@ -418,81 +422,133 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         // ring (and loads the shared-memory owner tiles first), warp 2 the L ring.  Lane 0 issues the TMA
         // boxes of columns 0..63; all lanes copy the columns from 64 on, 16 bytes per row and chunk, and
         // signal them one tile later so that two tiles of copies are in flight.
-        const int ring = warp >> 1;
-        const int S = ring == 0 ? SE : SL;
-        const int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
-        const CUtensorMap* maps[2] = {ring == 0 ? &tm_s0 : &tm_s2, ring == 0 ? &tm_s1 : &tm_s3};
-        const __nv_bfloat16* srcs[2] = {p.strm[2 * ring], p.strm[2 * ring + 1]};
+        // The element-wise warps leave these warps one issue slot in ten or so, and a stage is refilled no
+        // faster than this loop runs, so it is kept to a few dozen instructions per tile: everything that
+        // does not depend on the tile (lane's row, chunk positions, source pointers) is set up before it.
+        constexpr int KT = NA == 2 ? (DP - 64) / 8 : 1;  // 16-byte chunks per row behind column 64, at most
         const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
-        if (NPAIR == 2 && ring == 0) {
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
-                ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
-                ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
-            }
-            if constexpr (NA == 2) {
-                for (int i = lane; i < 2 * BWD_ROWS * ntail; i += 32) {
-                    const int t = i / (BWD_ROWS * ntail), rem = i - t * (BWD_ROWS * ntail);
-                    const int r = rem / ntail, k = rem - r * ntail;
-                    const bool v = row0 + r < p.N;
-                    const __nv_bfloat16* src = p.own[2 + t] + ((size_t)bh * p.N + (v ? row0 + r : 0)) * p.d + 64 + 8 * k;
-                    ptx::cp_async_16(own_base + t * C::OWN_BYTES + BWD_ROWS * 128 + k * BWD_ROWS * 16 + r * 16, src, v ? 16u : 0u);
+        const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
+        const int d32 = 32 * p.d;                                      // 32 rows further down, in elements
+        bool owner_pend = false;  // owner-tile copies issued (warp 0) and not signalled yet
+        auto produce = [&](auto ring_tag) -> void {
+            constexpr int ring = decltype(ring_tag)::value;
+            constexpr int S = ring == 0 ? SE : SL;
+            constexpr int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
+            constexpr uint32_t TB = ring == 0 ? C::EST_BYTES : C::LST_BYTES;
+            const CUtensorMap* map0 = ring == 0 ? &tm_s0 : &tm_s2;
+            const CUtensorMap* map1 = ring == 0 ? &tm_s1 : &tm_s3;
+            const uint32_t ring_base = ring == 0 ? e_base : l_base;
+            const __nv_bfloat16* base0 = p.strm[2 * ring];
+            const __nv_bfloat16* base1 = p.strm[2 * ring + 1];
+            [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
+            [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
+            [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
+            // Destination of chunk 0 of row `lane` behind the 64-column atom: the E ring keeps compact
+            // 16-byte-per-row blocks (K-major operands only), the L ring a second 128-byte-swizzled atom.
+            [[maybe_unused]] const uint32_t dst_lane = BC * 128 + (ring == 0 ? lane * 16 : lane * 128);
+            [[maybe_unused]] const uint32_t sw = lane & 7;  // rows 32 apart share it
+            bool ok = true;
+            int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
+            for (int j = 0; j < T; ++j) {
+                if constexpr (NA == 2) {
+                    // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
+                    // that tile before it frees the stage.
+                    if (pend_s >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
+                        ptx::cp_async_wait<0>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                        if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 3);
+                        pend_s = -1;
+                        if (ring == 0 && owner_pend) {  // cp.async groups complete in order: the owner copies have landed too
+                            if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+                            owner_pend = false;
+                        }
+                    }
                 }
-                ptx::cp_async_commit();
-                ptx::cp_async_wait<0>();
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+                ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                if (!ok) break;
+                if (lane == 0 && ring == 0) BTL_STAMP(2, j, 0);
+                const uint32_t stage = ring_base + s * 2 * TB;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
+                    ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
+                    ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
+                }
+                if constexpr (NA == 2) {
+                    const int rows_left = p.N - j * BC;  // rows of this tile that exist
+#pragma unroll
+                    for (int k = 0; k < KT; ++k) {
+                        if (k < ntail) {
+#pragma unroll
+                            for (int rp = 0; rp < BC / 32; ++rp) {
+                                const bool v = lane + 32 * rp < rows_left;
+                                const uint32_t dst = stage + dst_lane +
+                                                     (ring == 0 ? k * BC * 16 + rp * 32 * 16 : rp * 32 * 128 + ((k ^ sw) << 4));
+                                ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
+                                ptx::cp_async_16(dst + TB, v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                            }
+                        }
+                    }
+                    ptx::cp_async_commit();
+                    if (lane == 0 && ring == 0) BTL_STAMP(2, j, 1);
+                    if (pend_s >= 0) {  // the tile before: its copies have had a whole iteration to land
+                        ptx::cp_async_wait<1>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                        if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 2);
+                        if (ring == 0 && owner_pend) {
+                            if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+                            owner_pend = false;
+                        }
+                    }
+                    pend_s = s;
+                    src0 += tile_elems;
+                    src1 += tile_elems;
+                }
+                if (++s == S) { s = 0; ph ^= 1; }
             }
-        }
-        bool ok = true;
-        int pending = -1;  // tile whose copied columns have not been signalled yet
-        for (int j = 0; j < T; ++j) {
-            const int s = j % S, ph = (j / S) & 1;
-            if constexpr (NA == 2) {
-                // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
-                // that tile before it frees the stage.
-                if (pending >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
-                    ptx::cp_async_wait<0>();
+            if (NA == 2) {
+                ptx::cp_async_wait<0>();  // nothing of ours stays in flight
+                if (ok && pend_s >= 0) {
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(b_full + pending % S));
-                    pending = -1;
+                    if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                    if (ring == 0 && owner_pend && lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
                 }
             }
-            ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
-            if (!ok) break;
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
-                for (int t = 0; t < 2; ++t) ptx::tma_load_3d(tile_addr(2 * ring + t, j), maps[t], bar(b_full + s), 0, j * BC, bh);
-            }
-            if constexpr (NA == 2) {
-                for (int i = lane; i < 2 * BC * ntail; i += 32) {
-                    const int t = i / (BC * ntail), rem = i - t * (BC * ntail);
-                    const int r = rem / ntail, k = rem - r * ntail;
-                    const int grow = j * BC + r;
-                    const bool v = grow < p.N;
-                    const __nv_bfloat16* src = srcs[t] + ((size_t)bh * p.N + (v ? grow : 0)) * p.d + 64 + 8 * k;
-                    const uint32_t tail = tile_addr(2 * ring + t, j) + BC * 128;
-                    ptx::cp_async_16(ring == 0 ? tail + k * BC * 16 + r * 16 : tail + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+        };
+        if (warp == 0) {
+            if constexpr (NPAIR == 2) {
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
+                    ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
+                    ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
                 }
-                ptx::cp_async_commit();
-                if (pending >= 0) {  // the tile before: its copies have had a whole iteration to land
-                    ptx::cp_async_wait<1>();
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(b_full + pending % S));
+                if constexpr (NA == 2) {
+                    const __nv_bfloat16* o2 = p.own[2] + lane_row + (size_t)row0 * p.d;
+                    const __nv_bfloat16* o3 = p.own[3] + lane_row + (size_t)row0 * p.d;
+                    const int rows_left = p.N - row0;
+#pragma unroll
+                    for (int k = 0; k < KT; ++k) {
+                        if (k < ntail) {
+#pragma unroll
+                            for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
+                                const bool v = lane + 32 * rp < rows_left;
+                                const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
+                                ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[2], v ? 16u : 0u);
+                                ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[3], v ? 16u : 0u);
+                            }
+                        }
+                    }
+                    ptx::cp_async_commit();
+                    owner_pend = true;  // signalled with the first tile's copies: nothing needs them earlier
                 }
-                pending = j;
             }
-        }
-        if (NA == 2) {
-            ptx::cp_async_wait<0>();  // nothing of ours stays in flight
-            if (ok && pending >= 0) {
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar(b_full + pending % S));
-            }
+            produce(std::integral_constant<int, 0>{});
+        } else {
+            produce(std::integral_constant<int, 1>{});
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer: the whole warp runs

@@ -35,6 +35,7 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
+#include <type_traits>
 
 #include "sm100_ptx.cuh"
 
@@ -384,46 +385,89 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // end of a 144-byte row would read the next row's bytes from L2 only to replace them by zeros,
         // which nearly doubled the L2 traffic), and signal them one tile later so that two tiles of copies
         // are in flight.
-        const int ring = warp >> 1;
-        const int S = ring == 0 ? SE : SL;
-        const int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
-        const CUtensorMap* maps[2] = {ring == 0 ? &tm_k : &tm_v, ring == 0 ? &tm_tk : &tm_tv};
-        const __nv_bfloat16* srcs[2] = {ring == 0 ? p.K : p.V, ring == 0 ? p.tK : p.tV};
-        const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
-        bool ok = true;
-        for (int j = 0; j < T; ++j) {
-            const int s = j % S, ph = (j / S) & 1;
-            ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            if (!ok) break;
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
-                for (int t = 0; t < 2; ++t) ptx::tma_load_3d(tile_addr(2 * ring + t, j), maps[t], bar(b_full + s), 0, j * BC, bh);
-            }
-            if constexpr (NA == 2) {
-                for (int i = lane; i < 2 * BC * ntail; i += 32) {
-                    const int t = i / (BC * ntail), rem = i - t * (BC * ntail);
-                    const int r = rem / ntail, k = rem - r * ntail;
-                    const int grow = j * BC + r;
-                    const bool v = grow < p.N;
-                    const __nv_bfloat16* src = srcs[t] + ((size_t)bh * p.N + (v ? grow : 0)) * p.d + 64 + 8 * k;
-                    ptx::cp_async_16(tile_addr(2 * ring + t, j) + BC * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+        // The element-wise warps leave these warps one issue slot in ten or so, and a stage is refilled no
+        // faster than this loop runs, so it is kept to a few dozen instructions per tile: everything that
+        // does not depend on the tile (lane's row, chunk positions, source pointers) is set up before it.
+        constexpr int KT = NA == 2 ? (DP - 64) / 8 : 1;  // 16-byte chunks per row behind column 64, at most
+        [[maybe_unused]] const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
+        [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
+        [[maybe_unused]] const int d32 = 32 * p.d;                                      // 32 rows further down, in elements
+        auto produce = [&](auto ring_tag) -> void {
+            constexpr int ring = decltype(ring_tag)::value;
+            constexpr int S = ring == 0 ? SE : SL;
+            constexpr int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
+            constexpr uint32_t TB = C::ST_BYTES;
+            const CUtensorMap* map0 = ring == 0 ? &tm_k : &tm_v;
+            const CUtensorMap* map1 = ring == 0 ? &tm_tk : &tm_tv;
+            const uint32_t ring_base = ring == 0 ? e_base : l_base;
+            const __nv_bfloat16* base0 = ring == 0 ? p.K : p.V;
+            const __nv_bfloat16* base1 = ring == 0 ? p.tK : p.tV;
+            [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
+            [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
+            [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
+            // chunk k of row r behind the 64-column atom sits at physical chunk k ^ (r & 7) of a second atom
+            [[maybe_unused]] const uint32_t dst_lane = BC * 128 + lane * 128;
+            [[maybe_unused]] const uint32_t sw = lane & 7;  // rows 32 apart share it
+            bool ok = true;
+            int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
+            for (int j = 0; j < T; ++j) {
+                if constexpr (NA == 2) {
+                    // Do not sit on a tile's unsignalled copies while waiting for a free stage: its consumer
+                    // could be using the time.
+                    if (pend_s >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
+                        ptx::cp_async_wait<0>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                        pend_s = -1;
+                    }
                 }
-                ptx::cp_async_commit();
-                if (j > 0) {
-                    ptx::cp_async_wait<1>();
+                ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS);
+                if (!ok) break;
+                const uint32_t stage = ring_base + s * 2 * TB;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
+                    ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
+                    ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
+                }
+                if constexpr (NA == 2) {
+                    const int rows_left = p.N - j * BC;  // keys of this tile that exist
+#pragma unroll
+                    for (int k = 0; k < KT; ++k) {
+                        if (k < ntail) {
+#pragma unroll
+                            for (int rp = 0; rp < BC / 32; ++rp) {
+                                const bool v = lane + 32 * rp < rows_left;
+                                const uint32_t dst = stage + dst_lane + rp * 32 * 128 + ((k ^ sw) << 4);
+                                ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
+                                ptx::cp_async_16(dst + TB, v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                            }
+                        }
+                    }
+                    ptx::cp_async_commit();
+                    if (pend_s >= 0) {  // the tile before: its copies have had a whole iteration to land
+                        ptx::cp_async_wait<1>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                    }
+                    pend_s = s;
+                    src0 += tile_elems;
+                    src1 += tile_elems;
+                }
+                if (++s == S) { s = 0; ph ^= 1; }
+            }
+            if (NA == 2) {
+                ptx::cp_async_wait<0>();  // nothing of ours stays in flight
+                if (ok && pend_s >= 0) {
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(b_full + (j - 1) % S));
+                    if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
                 }
             }
-        }
-        if (NA == 2 && ok) {
-            ptx::cp_async_wait<0>();
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(b_full + (T - 1) % S));
-        }
-        if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
+        };
+        if (warp == 0) produce(std::integral_constant<int, 0>{});
+        else produce(std::integral_constant<int, 1>{});
     } else if (warp == 1) {
         // ------------------------------------------------------------------ score MMAs (warp 1) and value MMAs
         // (warp 3), on two schedulers: an MMA costs 7 to 14 issue slots of its scheduler, which the element-wise
