@@ -45,8 +45,6 @@ enum : int { BWD_DV = 0, BWD_DK = 1, BWD_DQ = 2 };
 
 constexpr int BWD_THREADS = 640;  // 4 control warps + 16 element-wise warps
 constexpr int BWD_ROWS = 128;     // owner rows per CTA
-constexpr int BWD_STATS_STAGES = 8;  // ring of per-query statistics tiles
-constexpr int BWD_STATS_LAG = 3;     // statistics copies in flight
 constexpr uint64_t BWD_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;
 
 struct BwdParams {
@@ -103,6 +101,9 @@ struct BwdCfg {
     static constexpr int SL = NA == 1 ? 4 : 3;
     static constexpr int TILE_BYTES = NOWN_SMEM * OWN_BYTES + SE * 2 * EST_BYTES + SL * 2 * LST_BYTES;
     static constexpr int FULL_COUNT = NA;                  // TMA issuer (+ the warp copying columns >= 64)
+    // The L-ring producer also copies the per-query statistics of a tile (transposed passes), into a slot
+    // that lives and dies with the tile's L stage.
+    static constexpr int LFULL_COUNT = (NA == 2 || TRANSPOSED) ? 2 : 1;
     // which ring holds what: the E ring is released after the score MMAs, the L ring after the output MMAs.
     // DV: E = (Q, tQ) score operands, L = (Hc, G) output operands.
     // DK, DQ: E = second-pair score operands (Hc, G | V, tV), L = first-pair score operands that are also
@@ -117,11 +118,9 @@ struct BwdCfg {
     static constexpr int B_FINAL = B_PREADY + 2;
     static constexpr int B_QREADY = B_FINAL + 1;
     static constexpr int B_OWNER = B_QREADY + 1;
-    static constexpr int B_STFULL = B_OWNER + 1;
-    static constexpr int B_STEMPTY = B_STFULL + BWD_STATS_STAGES;
-    static constexpr int NBARS = B_STEMPTY + BWD_STATS_STAGES;
+    static constexpr int NBARS = B_OWNER + 1;
     static_assert(NBARS <= 48, "barrier table too small");
-    static constexpr int STATS_FLOATS = BWD_STATS_STAGES * 4 * 64;
+    static constexpr int STATS_FLOATS = SL * 4 * 64;
     static constexpr int MISC_BYTES = 48 * 8 + 64 + STATS_FLOATS * 4;
     static constexpr int SMEM_BYTES = TILE_BYTES + MISC_BYTES + 1024 /*alignment slack*/;
     // TMEM columns: accumulators, the bf16 owner operands X0, X1 in the gaps behind them, two score buffers
@@ -192,10 +191,11 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     for (int j = 0; j < T; ++j) {
         const int b = NPAIR == 1 ? (j & 1) : 0, sph = NPAIR == 1 ? (j >> 1) & 1 : (j & 1);
         if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        const float* st = stats + (j % BWD_STATS_STAGES) * 4 * 64 + 16 * sl;
+        // the statistics of the tile's queries arrive with its L stage, which is not released before the
+        // output MMAs of this tile, hence not before every warp is through with them
+        const float* st = stats + (j % C::SL) * 4 * 64 + 16 * sl;
         if (C::TRANSPOSED)
-            if (!ptx::mbar_wait(bar(C::B_STFULL + j % BWD_STATS_STAGES), (j / BWD_STATS_STAGES) & 1, abort_flag,
-                                BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            if (!ptx::mbar_wait(bar(C::B_LFULL + j % C::SL), (j / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 0);
         const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
@@ -302,10 +302,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         __syncwarp();
         if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);
         if (lane == 0) BTL_STAMP(4 + (w >> 3), j, w & 7);
-        if (lane == 0) {
-            ptx::mbar_arrive(bar(C::B_PREADY + b));
-            if (C::TRANSPOSED) ptx::mbar_arrive(bar(C::B_STEMPTY + j % BWD_STATS_STAGES));
-        }
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
     }
     if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, BWD_WAIT_LIMIT_NS);
     if (ok) {
@@ -366,7 +363,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
-        for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
+        for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::LFULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar(C::B_SFULL + b), 1);
             ptx::mbar_init(bar(C::B_PREADY + b), BC / 4);  // one arrival per warp working on a tile
@@ -374,10 +371,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         ptx::mbar_init(bar(C::B_FINAL), 1);
         ptx::mbar_init(bar(C::B_QREADY), 16);
         ptx::mbar_init(bar(C::B_OWNER), C::FULL_COUNT);
-        for (int s = 0; s < BWD_STATS_STAGES; ++s) {
-            ptx::mbar_init(bar(C::B_STFULL + s), 1);
-            ptx::mbar_init(bar(C::B_STEMPTY + s), BC / 4);
-        }
         ptx::fence_mbar_init();
     }
     if (NA == 2) {
@@ -435,6 +428,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             constexpr int S = ring == 0 ? SE : SL;
             constexpr int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
             constexpr uint32_t TB = ring == 0 ? C::EST_BYTES : C::LST_BYTES;
+            constexpr bool STATS = ring == 1 && C::TRANSPOSED;  // this ring carries the per-query statistics
+            constexpr bool HAS_CP = NA == 2 || STATS;           // the warp copies something itself
+            constexpr int NST = 2 * NPAIR;                      // statistics per query: lse2, mu (, Sigma1, c)
             const CUtensorMap* map0 = ring == 0 ? &tm_s0 : &tm_s2;
             const CUtensorMap* map1 = ring == 0 ? &tm_s1 : &tm_s3;
             const uint32_t ring_base = ring == 0 ? e_base : l_base;
@@ -447,10 +443,16 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // 16-byte-per-row blocks (K-major operands only), the L ring a second 128-byte-swizzled atom.
             [[maybe_unused]] const uint32_t dst_lane = BC * 128 + (ring == 0 ? lane * 16 : lane * 128);
             [[maybe_unused]] const uint32_t sw = lane & 7;  // rows 32 apart share it
+            // statistics: 16-byte chunks when the rows of the (B, H, N) arrays are 16-byte aligned, else floats
+            const bool st16 = (p.N & 3) == 0;
+            [[maybe_unused]] const uint32_t st_base = ptx::smem_u32(stats);
+            [[maybe_unused]] const size_t srow = (size_t)bh * p.N;
+            [[maybe_unused]] const float* st_src0 = (lane < 16 ? p.lse2 : p.mu) + srow + 4 * (lane & 15);
+            [[maybe_unused]] const float* st_src1 = NST == 4 ? (lane < 16 ? p.sig1 : p.cvec) + srow + 4 * (lane & 15) : nullptr;
             bool ok = true;
             int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
             for (int j = 0; j < T; ++j) {
-                if constexpr (NA == 2) {
+                if constexpr (HAS_CP) {
                     // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
                     // that tile before it frees the stage.
                     if (pend_s >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
@@ -475,10 +477,27 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
                     ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
                 }
-                if constexpr (NA == 2) {
-                    const int rows_left = p.N - j * BC;  // rows of this tile that exist
+                if constexpr (HAS_CP) {
+                    [[maybe_unused]] const int rows_left = p.N - j * BC;  // rows of this tile that exist
+                    if constexpr (STATS) {
+                        // queries beyond N read as zero: their rows of the B operands are zero too
+                        const uint32_t slot = st_base + s * (4 * 64 * 4);
+                        if (st16) {
+                            const bool v = 4 * (lane & 15) < rows_left;
+                            const uint32_t dst = slot + (lane >> 4) * 256 + (lane & 15) * 16;
+                            ptx::cp_async_16(dst, v ? st_src0 + j * BC : p.lse2, v ? 16u : 0u);
+                            if (NST == 4) ptx::cp_async_16(dst + 512, v ? st_src1 + j * BC : p.lse2, v ? 16u : 0u);
+                        } else {
+                            for (int c = lane; c < NST * 64; c += 32) {
+                                const int stat = c >> 6, r = c & 63;
+                                const float* src = (stat == 0 ? p.lse2 : stat == 1 ? p.mu : stat == 2 ? p.sig1 : p.cvec) + srow + j * BC + r;
+                                const bool v = r < rows_left;
+                                ptx::cp_async_4(slot + c * 4, v ? src : p.lse2, v ? 4u : 0u);
+                            }
+                        }
+                    }
 #pragma unroll
-                    for (int k = 0; k < KT; ++k) {
+                    for (int k = 0; k < (NA == 2 ? KT : 0); ++k) {
                         if (k < ntail) {
 #pragma unroll
                             for (int rp = 0; rp < BC / 32; ++rp) {
@@ -504,12 +523,14 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         }
                     }
                     pend_s = s;
-                    src0 += tile_elems;
-                    src1 += tile_elems;
+                    if constexpr (NA == 2) {
+                        src0 += tile_elems;
+                        src1 += tile_elems;
+                    }
                 }
                 if (++s == S) { s = 0; ph ^= 1; }
             }
-            if (NA == 2) {
+            if (HAS_CP) {
                 ptx::cp_async_wait<0>();  // nothing of ours stays in flight
                 if (ok && pend_s >= 0) {
                     ptx::fence_proxy_async_smem();
@@ -726,55 +747,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
         }
     } else if (warp == 3) {
-        // ------------------------------------------------------------------ per-query statistics (transposed passes):
-        // lse2, mu (and Sigma1, c for DK) of the tile's queries, copied asynchronously into a ring so that
-        // their latency (about a microsecond per global load) stays off the tile loop.
-        if (C::TRANSPOSED) {
-            const size_t srow = (size_t)bh * p.N;
-            const float* src_stat[4] = {p.lse2, p.mu, p.sig1, p.cvec};
-            if ((p.N & 3) == 0) {
-                constexpr int CPS = BC / 4;  // 16-byte chunks per statistic and tile
-                bool ok = true;
-                for (int j = 0; j < T; ++j) {
-                    const int s = j % BWD_STATS_STAGES, ph = (j / BWD_STATS_STAGES) & 1;
-                    ok = ptx::mbar_wait_warp(bar(C::B_STEMPTY + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                    if (!ok) break;
-#pragma unroll
-                    for (int i = lane; i < 2 * NPAIR * CPS; i += 32) {
-                        const int stat = i / CPS, chunk = i - stat * CPS;
-                        const bool v = j * BC + 4 * chunk < p.N;  // queries beyond N read as zero: their B rows are zero too
-                        ptx::cp_async_16(ptx::smem_u32(stats + s * 4 * 64 + stat * 64 + 4 * chunk),
-                                         src_stat[stat] + srow + (v ? j * BC + 4 * chunk : 0), v ? 16u : 0u);
-                    }
-                    ptx::cp_async_commit();
-                    if (j >= BWD_STATS_LAG) {
-                        ptx::cp_async_wait<BWD_STATS_LAG>();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(bar(C::B_STFULL + (j - BWD_STATS_LAG) % BWD_STATS_STAGES));
-                    }
-                }
-                ptx::cp_async_wait<0>();
-                __syncwarp();
-                if (ok && lane == 0)
-                    for (int j = (T > BWD_STATS_LAG ? T - BWD_STATS_LAG : 0); j < T; ++j)
-                        ptx::mbar_arrive(bar(C::B_STFULL + j % BWD_STATS_STAGES));
-            } else {
-                // rows of the statistics are not 16-byte aligned for this N: plain loads, one tile at a time
-                for (int j = 0; j < T; ++j) {
-                    const int s = j % BWD_STATS_STAGES, ph = (j / BWD_STATS_STAGES) & 1;
-                    if (!ptx::mbar_wait_warp(bar(C::B_STEMPTY + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS)) break;
-                    float* st = stats + s * 4 * 64;
-                    for (int c = lane; c < BC; c += 32) {
-                        const int i = j * BC + c;
-                        const bool v = i < p.N;
-#pragma unroll
-                        for (int k = 0; k < 2 * NPAIR; ++k) st[k * 64 + c] = v ? src_stat[k][srow + i] : 0.f;
-                    }
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(C::B_STFULL + s));
-                }
-            }
-        }
+        // idle
     } else {
         bwd_elementwise<MODE, DP>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, bh, row0, T);
     }
