@@ -158,7 +158,12 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     constexpr int BC = C::BC, KS = C::KS, NPAIR = C::NPAIR;
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
     const int q = w & 3, slot = w >> 2;
-    const int sl = slot;  // 16-column slice of every tile = one k-step of the output GEMMs
+    // DK, DQ: every warp works on every tile, on the 16-column slice `slot` (one k-step of the output GEMMs).
+    // DV (two score buffers): the warps split by tile parity, eight per tile, two slices each.  A warp then
+    // waits half as often for twice the work, and while the eight of one tile wait for their scores the other
+    // eight compute: with all sixteen on one tile the issue ports idled through every hand-off.
+    const int par = NPAIR == 1 ? (w >> 3) : 0, jstep = NPAIR == 1 ? 2 : 1;
+    const int sl = NPAIR == 1 ? 2 * (slot & 1) : slot;  // first (or only) slice of this warp
     const int row = q * 32 + lane;  // owner row inside the CTA tile
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const bool row_valid = row0 + row < p.N;
@@ -188,7 +193,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         r_cv = p.cvec[grow];
     }
     bool ok = true;
-    for (int j = 0; j < T; ++j) {
+    for (int j = par; j < T; j += jstep) {
         const int b = NPAIR == 1 ? (j & 1) : 0, sph = NPAIR == 1 ? (j >> 1) & 1 : (j & 1);
         if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
         // the statistics of the tile's queries arrive with its L stage, which is not released before the
@@ -201,16 +206,20 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
         const int key0 = j * BC + 16 * sl;  // first stream row of this slice
         if (NPAIR == 1) {
+          const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {  // this warp's two slices
+            const uint32_t sb = sbase + 16 * sub;
+            const float* stt = st + 16 * sub;
             uint32_t s1[16], s2[16];
-            ptx::tmem_ld16(sbase, s1);
-            ptx::tmem_ld16(sbase + BC, s2);
+            ptx::tmem_ld16(sb, s1);
+            ptx::tmem_ld16(sb + BC, s2);
             ptx::tmem_wait_ld();
             uint32_t pa0[8], pa1[8];
-            const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
 #pragma unroll
             for (int c4 = 0; c4 < 16; c4 += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
-                const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
+                const float4 l4 = *reinterpret_cast<const float4*>(stt + c4);
+                const float4 m4 = *reinterpret_cast<const float4*>(stt + 64 + c4);
                 const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
                 for (int e = 0; e < 4; e += 2) {  // P = 2^(c2 s - lse2), P Nn with Nn = alpha ts - mu: two columns per instruction
@@ -226,9 +235,10 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     pa1[(c4 + e) >> 1] = ptx::pack_bf16(q0, q1);
                 }
             }
-            // operand of k-step sl (16 stream rows) sits at column 16*sl of the accumulator it replaces
-            ptx::tmem_st8(sbase, pa0);
-            ptx::tmem_st8(sbase + BC, pa1);
+            // operand of a k-step (16 stream rows) sits at the slice's columns of the accumulator it replaces
+            ptx::tmem_st8(sb, pa0);
+            ptx::tmem_st8(sb + BC, pa1);
+          }
         } else {
             // ---- phase A: P, Nn, -P Sigma1, -P c from (S, Sd), two columns per register pair; then that half of the
             // buffer may be overwritten.  Phase B, which sits on the critical path between the second score pair and
@@ -351,6 +361,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     const uint32_t bar0 = ptx::smem_u32(misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48 * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 48 * 8 + 16);
+    const uint32_t turn_addr = bar0 + 48 * 8 + 32;  // turn counter of the two MMA issuers
     float* stats = reinterpret_cast<float*>(misc + 48 * 8 + 64);  // [stage][4][64]
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
 
@@ -362,11 +373,12 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
+        *reinterpret_cast<volatile uint32_t*>(misc + 48 * 8 + 32) = 0u;
         for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
         for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::LFULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar(C::B_SFULL + b), 1);
-            ptx::mbar_init(bar(C::B_PREADY + b), BC / 4);  // one arrival per warp working on a tile
+            ptx::mbar_init(bar(C::B_PREADY + b), NPAIR == 1 ? 8 : 16);  // one arrival per warp working on a tile
         }
         ptx::mbar_init(bar(C::B_FINAL), 1);
         ptx::mbar_init(bar(C::B_QREADY), 16);
@@ -571,9 +583,17 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         } else {
             produce(std::integral_constant<int, 1>{});
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer: the whole warp runs
-        // the loop in converged control flow; one elected lane issues (see mma_ts_elect)
+    } else if (warp == 1 || warp == 3) {
+        // ------------------------------------------------------------------ MMA issuers, warps 1 and 3: each
+        // whole warp runs its loop in converged control flow; one elected lane issues (see mma_ts_elect).
+        // An issuing thread is held at the rate of the tensor pipe while its MMAs are queued, and the waits
+        // and address arithmetic between two steps cost it several hundred clocks next to the element-wise
+        // warps of its scheduler; with one issuer that time is added to every tile.  DV: warp 1 takes the
+        // even tiles (score buffer 0), warp 3 the odd ones; a tile's output MMAs and the score MMAs that
+        // overwrite their operands come from one thread, so the pipe orders them; the accumulating output
+        // MMAs of consecutive tiles are ordered by a turn counter.  DK, DQ: warp 1 alone; their one score
+        // buffer already serialises the steps.
+        const int wsel = warp >> 1;  // 0: warp 1, 1: warp 3
         constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
         constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
@@ -590,17 +610,12 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             return kk < 4 ? ptx::smem_desc_sw128(base, 16, 1024) + (uint64_t)((kk * 32) >> 4)
                           : ptx::smem_desc_nosw(base + BWD_ROWS * 128, BWD_ROWS * 16, 128);
         };
-        // `ready`: the caller has already seen every barrier of this step complete (mbar_test3_warp)
-        auto issue_scores = [&](int j, bool ready) -> bool {
+        auto issue_scores = [&](int j, bool) -> bool {
             const int b = j & 1;
-            if (!ready) {
-                if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-                if (NPAIR == 2)
-                    if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-            }
+            if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
             if (lane == 0) BTL_STAMP(0, j, 0);
-            // DV only (the two-pair passes use the split-phase loop below): Y0, Y1 in the E ring, K-major B
+            // DV only (the two-pair passes have their own loops below): Y0, Y1 in the E ring, K-major B
             const uint32_t t0 = tile_addr(0, j), t1 = tile_addr(1, j);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
 #pragma unroll
@@ -617,15 +632,14 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             if (lane == 0) BTL_STAMP(0, j, 1);
             return true;
         };
-        auto issue_outputs = [&](int j, bool ready) -> bool {
+        auto issue_outputs = [&](int j, bool) -> bool {  // DV only
             const int b = j & 1;
             if (lane == 0) BTL_STAMP(0, j, 2);
-            if (!ready) {
-                if (NPAIR == 1)
-                    if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-                if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-                ptx::tc_fence_after_sync();
-            }
+            if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            // the other issuer has queued its batch of tile j - 1: accumulation order is the tile order
+            if (!ptx::turn_wait_warp(turn_addr, (uint32_t)j, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            ptx::tc_fence_after_sync();
             if (lane == 0) BTL_STAMP(0, j, 3);
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B (the L ring): atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
@@ -646,108 +660,109 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             return true;
         };
         bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-        if (ok && NPAIR == 2) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), 0, abort_flag, BWD_WAIT_LIMIT_NS);
         ptx::tc_fence_after_sync();
         if constexpr (NPAIR == 1) {
-            if (ok) ok = issue_scores(0, false);
-            for (int j = 0; ok && j < T; ++j) {
-                // one combined poll of what the two steps below wait for
-                bool ready = false;
-                if (j + 1 < T) {
-                    const int jn = j + 1;
-                    ready = ptx::mbar_test3_warp(bar(C::B_EFULL + jn % SE), (jn / SE) & 1, bar(C::B_LFULL + j % SL), (j / SL) & 1,
-                                                 bar(C::B_PREADY + (j & 1)), (j >> 1) & 1);
-                    ok = issue_scores(jn, ready);
-                }
-                if (ok) ok = issue_outputs(j, ready);
+            // warp `wsel` owns the tiles j = wsel, wsel + 2, ...: S(j), then per tile outputs(j) and S(j + 2)
+            if (ok && wsel < T) ok = issue_scores(wsel, false);
+            // The turn passes on after the whole batch (outputs(j), S(j + 2)): two batches queued at once
+            // would share the pipe MMA by MMA, both would finish late and together, and the element-wise
+            // work of the two buffers would then run back to back instead of under the other's MMAs.
+            for (int j = wsel; ok && j < T; j += 2) {
+                ok = issue_outputs(j, false);  // waits for the L tile, the operands and its turn
+                if (ok && j + 2 < T) ok = issue_scores(j + 2, false);
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)j + 1u);
             }
         } else {
-            // One score buffer used in two phases.  Order on the tensor pipe:
-            //   (S, Sd)(0), (D, X)(0), then per tile j: (S, Sd)(j+1) once the element-wise warps have read
-            //   (S, Sd)(j) | outputs(j) once the operands W, dA are written | (D, X)(j+1), which overwrites them.
-            const uint32_t dS = tb + C::COL_SCORE, dT = dS + BC, dD = dS + 2 * BC, dX = dS + 3 * BC;
-            auto issue_first_pair = [&](int j) {  // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; Y0, Y1 in the L ring, K-major
-                const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, j), 16, 1024);
-                const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, j), 16, 1024);
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ts_elect(dS, ax0 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
-                }
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ts_elect(dT, ax1 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
-                }
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                    ptx::mma_ts_elect(dT, ax0 + 8 * kk, y1 + off, idesc_s, 1u);
-                }
-                ptx::mma_commit_elect(bar(C::B_SFULL + 0));
-            };
-            auto issue_second_pair = [&](int j) {  // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; Y2, Y3 in the E ring
-                const uint32_t t2 = tile_addr(0, j), t3 = tile_addr(1, j);
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dD, own_kdesc(0, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(1, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
-#pragma unroll
-                for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(0, kk), e_kdesc(t3, kk), idesc_s, 1u);
-                ptx::mma_commit_elect(bar(C::B_SFULL + 1));
-                ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
-            };
-            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-            if (ok) {
+            if (wsel == 0) {  // one issuer: splitting these steps over two warps measured 1 to 2 % slower
+                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), 0, abort_flag, BWD_WAIT_LIMIT_NS);
                 ptx::tc_fence_after_sync();
-                issue_first_pair(0);
-                issue_second_pair(0);
-            }
-            for (int j = 0; ok && j < T; ++j) {
-                if (j + 1 < T) {
-                    const int jn = j + 1;
-                    // (S, Sd)(j) read by all element-wise warps, and the tiles of j+1 loaded
-                    const bool ready = ptx::mbar_test3_warp(bar(C::B_PREADY + 1), j & 1, bar(C::B_LFULL + jn % SL), (jn / SL) & 1,
-                                                            bar(C::B_EFULL + jn % SE), (jn / SE) & 1);
-                    if (!ready) {
-                        ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                        if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + jn % SL), (jn / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                        if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + jn % SE), (jn / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                        if (!ok) break;
+                // One score buffer used in two phases.  Order on the tensor pipe:
+                //   (S, Sd)(0), (D, X)(0), then per tile j: (S, Sd)(j+1) once the element-wise warps have read
+                //   (S, Sd)(j) | outputs(j) once the operands W, dA are written | (D, X)(j+1), which overwrites them.
+                const uint32_t dS = tb + C::COL_SCORE, dT = dS + BC, dD = dS + 2 * BC, dX = dS + 3 * BC;
+                auto issue_first_pair = [&](int j) {  // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; Y0, Y1 in the L ring, K-major
+                    const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, j), 16, 1024);
+                    const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, j), 16, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                        ptx::mma_ts_elect(dS, ax0 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
                     }
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                        ptx::mma_ts_elect(dT, ax1 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                        ptx::mma_ts_elect(dT, ax0 + 8 * kk, y1 + off, idesc_s, 1u);
+                    }
+                    ptx::mma_commit_elect(bar(C::B_SFULL + 0));
+                };
+                auto issue_second_pair = [&](int j) {  // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; Y2, Y3 in the E ring
+                    const uint32_t t2 = tile_addr(0, j), t3 = tile_addr(1, j);
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dD, own_kdesc(0, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(1, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(0, kk), e_kdesc(t3, kk), idesc_s, 1u);
+                    ptx::mma_commit_elect(bar(C::B_SFULL + 1));
+                    ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+                };
+                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+                if (ok) {
                     ptx::tc_fence_after_sync();
-                    if (lane == 0) BTL_STAMP(0, jn, 0);
-                    issue_first_pair(jn);
-                    if (lane == 0) BTL_STAMP(0, jn, 1);
+                    issue_first_pair(0);
+                    issue_second_pair(0);
                 }
-                // outputs(j): acc0 += W B0, acc1 += dA B0 + W B1 with the operands in the D and X columns
-                if (lane == 0) BTL_STAMP(0, j, 2);
-                ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                if (lane == 0) BTL_STAMP(0, j, 3);
-                {
-                    const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);  // MN-major B
-                    const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
-                    const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
-#pragma unroll
-                    for (int u = 0; u < BC / 16; ++u) {
-                        const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
-                        const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                        ptx::mma_ts_elect(acc0, dD + 16 * u, b0 + off, idesc_o, acc);
-                        ptx::mma_ts_elect(acc1, dX + 16 * u, b0 + off, idesc_o, acc);
-                        ptx::mma_ts_elect(acc1, dD + 16 * u, b1 + off, idesc_o, 1u);
+                for (int j = 0; ok && j < T; ++j) {
+                    if (j + 1 < T) {
+                        const int jn = j + 1;
+                        // (S, Sd)(j) read by all element-wise warps, and the tiles of j+1 loaded
+                        const bool ready = ptx::mbar_test3_warp(bar(C::B_PREADY + 1), j & 1, bar(C::B_LFULL + jn % SL), (jn / SL) & 1,
+                                                                bar(C::B_EFULL + jn % SE), (jn / SE) & 1);
+                        if (!ready) {
+                            ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + jn % SL), (jn / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + jn % SE), (jn / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                            if (!ok) break;
+                        }
+                        ptx::tc_fence_after_sync();
+                        if (lane == 0) BTL_STAMP(0, jn, 0);
+                        issue_first_pair(jn);
+                        if (lane == 0) BTL_STAMP(0, jn, 1);
                     }
-                    ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
-                    if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                    // outputs(j): acc0 += W B0, acc1 += dA B0 + W B1 with the operands in the D and X columns
+                    if (lane == 0) BTL_STAMP(0, j, 2);
+                    ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (lane == 0) BTL_STAMP(0, j, 3);
+                    {
+                        const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);  // MN-major B
+                        const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+                        const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+#pragma unroll
+                        for (int u = 0; u < BC / 16; ++u) {
+                            const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                            const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                            ptx::mma_ts_elect(acc0, dD + 16 * u, b0 + off, idesc_o, acc);
+                            ptx::mma_ts_elect(acc1, dX + 16 * u, b0 + off, idesc_o, acc);
+                            ptx::mma_ts_elect(acc1, dD + 16 * u, b1 + off, idesc_o, 1u);
+                        }
+                        ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+                        if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                    }
+                    if (lane == 0) BTL_STAMP(0, j, 4);
+                    if (j + 1 < T) issue_second_pair(j + 1);
                 }
-                if (lane == 0) BTL_STAMP(0, j, 4);
-                if (j + 1 < T) issue_second_pair(j + 1);
             }
         }
-    } else if (warp == 3) {
-        // idle
     } else {
         bwd_elementwise<MODE, DP>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, bh, row0, T);
     }

@@ -254,6 +254,35 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     return __all_sync(0xffffffffu, ok);
 }
 
+// A turn counter in shared memory orders steps of two warps: `turn_post` publishes a count, `turn_wait_warp`
+// waits (bounded like mbar_wait; warp-uniform result) until it has reached `want`.
+__device__ __forceinline__ void turn_post(uint32_t addr, uint32_t value) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(addr), "r"(value) : "memory");
+}
+__device__ __forceinline__ uint32_t turn_read(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ bool turn_wait_warp(uint32_t addr, uint32_t want, volatile int* abort_flag, uint64_t limit_ns) {
+    bool ok = true;
+    if (turn_read(addr) < want) {
+        const uint64_t t0 = globaltimer_ns();
+        for (uint32_t it = 1;; ++it) {
+            if (turn_read(addr) >= want) break;
+            if ((it & 255u) == 0u) {
+                if (*abort_flag) { ok = false; break; }
+                if (globaltimer_ns() - t0 > limit_ns) {
+                    *abort_flag = 1;
+                    ok = false;
+                    break;
+                }
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
 // Non-blocking test of one mbarrier phase; warp-uniform result.
 __device__ __forceinline__ bool mbar_test_warp(uint32_t bar, uint32_t parity) {
     uint32_t ok;
