@@ -10,22 +10,27 @@
 // with P = 2^(c2 S - lse2), Nn = alpha Sd - mu, W = P (D - Sigma1), dA = P (X - c) + W Nn, and
 //   acc0 += A0 B0,  acc1 += A1 B0 + A0 B1      (B0, B1 = Hc, G | Q, tQ | K, tK).
 //
-// A CTA owns 128 owner rows of one head and streams the other side in tiles of BC rows (64 for DV,
-// 32 for DK and DQ, whose four score accumulators need twice the tensor-memory columns).
+// A CTA owns 128 owner rows of one head and streams the other side in tiles of BC = 64 rows.
 //
 // What is where
 //   * The owner operands of the first score pair (K, tK or Q, tQ) are written once into tensor memory
 //     as bf16 A operands: with A in tensor memory a 128 x N x 16 MMA runs at full rate for N >= 32,
-//     while with A in shared memory it is bound by the shared-memory port (N = 32: 40 clk instead of 16).
+//     while with A in shared memory it is bound by the shared-memory port (N = 64: 48 clk instead of 32).
 //     The owner operands of the second score pair (V, tV or Hc, G) stay in shared memory: tensor
-//     memory has no room for them next to two score buffers.
-//   * Score accumulators are double-buffered; the bf16 operands A0, A1 are written back over the
-//     columns of the first two accumulators and consumed from tensor memory.
-//   * 16 element-wise warps: warp w works on TMEM lane quadrant w % 4 (32 owner rows) and on the
-//     slice w / 4 (BC / 4 columns) of every tile.  Nothing is exchanged between them.
+//     memory has no room for them next to the score accumulators.
+//   * Score accumulators: DV has two buffers of (S | Sd), so that the MMAs of one tile run under the
+//     element-wise work of the other; DK and DQ have one buffer of (S | Sd | D | X) used in two phases
+//     (S, Sd are turned into P, Nn in registers and their columns released while D, X are still being
+//     computed).  The bf16 operands A0, A1 are written back over accumulator columns the writing warp
+//     has read and are consumed from tensor memory by the output MMAs.
+//   * 16 element-wise warps: warp w works on TMEM lane quadrant w % 4 (32 owner rows).  DK, DQ: on the
+//     16-column slice w / 4 of every tile.  DV: the warps split by tile parity, eight per tile, two
+//     slices each.  Nothing is exchanged between them.
 //   * Streamed columns 0..63 arrive by TMA; columns from 64 on are 16-byte asynchronous copies (a
 //     64-column box hanging over the end of a 144-byte row would read the next row from L2 for nothing).
-//   * Per-query statistics of the transposed passes (DV, DK) are staged in shared memory by warp 3.
+//     The L-ring producer also copies the per-query statistics of a tile (transposed passes DV, DK).
+//   * MMAs are issued by warp 1 (DK, DQ) or by warps 1 and 3 on alternate tiles, ordered by a turn
+//     counter (DV).
 //
 // Every wait on an mbarrier is bounded; when one gives up the block records a time-out status and
 // all roles leave their loops.
@@ -43,7 +48,7 @@ namespace tvm_attn {
 
 enum : int { BWD_DV = 0, BWD_DK = 1, BWD_DQ = 2 };
 
-constexpr int BWD_THREADS = 640;  // 4 control warps + 16 element-wise warps
+constexpr int BWD_THREADS = 640;  // 2 producer + 2 MMA-issuing warps, 16 element-wise warps
 constexpr int BWD_ROWS = 128;     // owner rows per CTA
 constexpr uint64_t BWD_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;
 
@@ -286,12 +291,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 }
             }
             // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 2);
             if (!ptx::mbar_wait(bar(C::B_SFULL + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after_sync();
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 3);
             uint32_t s3[16], s4[16];
             ptx::tmem_ld16(sbase + 2 * BC, s3);
             ptx::tmem_ld16(sbase + 3 * BC, s4);
             ptx::tmem_wait_ld();
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 4);
             uint32_t pa0[8], pa1[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
@@ -304,10 +312,12 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 pa0[k] = ptx::pack_bf16(w0, w1);
                 pa1[k] = ptx::pack_bf16(d0, d1);
             }
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 5);
             ptx::tmem_st8(sbase + 2 * BC, pa0);
             ptx::tmem_st8(sbase + 3 * BC, pa1);
         }
         ptx::tmem_wait_st();
+        if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 6);
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);

@@ -61,24 +61,8 @@ struct FwdParams {
     float* lse;
     float* mu;
     int* status;  // device status word; non-zero makes the kernel a no-op
-    unsigned long long* tl;  // timeline builds only: clock stamps of one CTA
+    unsigned long long* tl;  // unused (timeline builds of other variants)
 };
-
-#ifdef TVM_ATTN_TIMELINE
-#ifndef TVM_ATTN_TIMELINE_CTA
-#define TVM_ATTN_TIMELINE_CTA 0  // the CTA whose clock stamps are recorded
-#endif
-#define FTL_STAMP(role, j, ev)                                                                         \
-    do {                                                                                                \
-        if (p.tl && blockIdx.x == TVM_ATTN_TIMELINE_CTA && (j) < 64) {                                  \
-            unsigned long long t_;                                                                      \
-            asm volatile("mov.u64 %0, %clock64;" : "=l"(t_));                                          \
-            p.tl[((role) * 64 + (j)) * 8 + (ev)] = t_;                                                  \
-        }                                                                                               \
-    } while (0)
-#else
-#define FTL_STAMP(role, j, ev) do {} while (0)
-#endif
 
 template <int DP>
 struct FwdCfg {
@@ -157,54 +141,31 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
         // S is complete before Sd: the row maxima are found and exchanged while the Sd MMAs still run
         if (!ptx::mbar_wait(bar(C::B_SFULL + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
-        if (lane == 0 && w == 0) FTL_STAMP(1, j, 0);
         const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS;
         uint32_t s[16], ts[16];
-        // Row maximum over the whole tile: every warp reads all four slices of S itself.  (Exchanging
-        // slice maxima through shared memory costs two more barrier round trips per tile, each some
-        // hundreds of clocks next to fifteen other busy warps; 48 more columns of tensor-memory loads
-        // and 24 more max instructions cost less.)  Its own slice stays in registers.
-        float mx;
-        {
-            uint32_t u[16], v[16];
-            ptx::tmem_ld16(sbase + 16 * sl, s);
-            ptx::tmem_ld16(sbase + 16 * ((sl + 1) & 3), u);
-            ptx::tmem_wait_ld();
-            const int left = p.N - j * BC;  // columns of this tile that are real keys
-            if (left < BC) {
+        ptx::tmem_ld16(sbase + 16 * sl, s);
+        ptx::tmem_wait_ld();
+        const int nvalid = p.N - j * BC - 16 * sl;  // columns of this slice that are real keys
+        if (nvalid < 16) {
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    if (16 * sl + c >= left) s[c] = __float_as_uint(-CUDART_INF_F);
-                    if (16 * ((sl + 1) & 3) + c >= left) u[c] = __float_as_uint(-CUDART_INF_F);
-                }
-            }
-            mx = ptx::max3(__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(u[0]));
-#pragma unroll
-            for (int c = 2; c < 16; c += 2) mx = ptx::max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-#pragma unroll
-            for (int c = 1; c < 15; c += 2) mx = ptx::max3(mx, __uint_as_float(u[c]), __uint_as_float(u[c + 1]));
-            mx = fmaxf(mx, __uint_as_float(u[15]));
-            ptx::tmem_ld16(sbase + 16 * ((sl + 2) & 3), u);
-            ptx::tmem_ld16(sbase + 16 * ((sl + 3) & 3), v);
-            ptx::tmem_wait_ld();
-            if (left < BC) {
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    if (16 * ((sl + 2) & 3) + c >= left) u[c] = __float_as_uint(-CUDART_INF_F);
-                    if (16 * ((sl + 3) & 3) + c >= left) v[c] = __float_as_uint(-CUDART_INF_F);
-                }
-            }
-#pragma unroll
-            for (int c = 0; c < 16; c += 2) mx = ptx::max3(mx, __uint_as_float(u[c]), __uint_as_float(u[c + 1]));
-#pragma unroll
-            for (int c = 0; c < 16; c += 2) mx = ptx::max3(mx, __uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+            for (int c = 0; c < 16; ++c)
+                if (c >= nvalid) s[c] = __float_as_uint(-CUDART_INF_F);
         }
-        if (lane == 0 && w == 0) FTL_STAMP(1, j, 1);
+        // slice maximum, exchanged with the three other warps of this quadrant
+        float mx = ptx::max3(__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(s[2]));
+#pragma unroll
+        for (int c = 3; c < 15; c += 2) mx = ptx::max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+        mx = fmaxf(mx, __uint_as_float(s[15]));
+        float* xm = xmax + (j & 1) * 512;
+        xm[row * 4 + sl] = mx;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_XMAX + q));
         if (!ptx::mbar_wait(bar(C::B_SFULL + 2 + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
-        if (lane == 0 && w == 0) FTL_STAMP(1, j, 2);
-        const float mrow = mx * p.c2;  // tile maximum of the row, log2 units
+        if (!ptx::mbar_wait(bar(C::B_XMAX + q), j & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        const float4 o4 = *reinterpret_cast<const float4*>(xm + row * 4);
+        const float mrow = fmaxf(ptx::max3(o4.x, o4.y, o4.z), o4.w) * p.c2;  // tile maximum of the row, log2 units
         ptx::tmem_wait_ld();
         const bool need = mrow > m_ref + FWD_LAZY_LOG2;
         if (__any_sync(0xffffffffu, need)) {
@@ -264,7 +225,6 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
                 }
             }
         }
-        if (lane == 0 && w == 0) FTL_STAMP(1, j, 3);
         // ---- P~ = 2^(c2 s - m), P~ (T - c); two elements per instruction where the hardware allows
         const uint64_t nm = ptx::pack2(-m_ref, -m_ref), nc = ptx::pack2(-cen, -cen);
         uint32_t pp[8], ppt[8];
@@ -290,11 +250,8 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0 && w == 0) FTL_STAMP(1, j, 4);
-        if (lane == 0) FTL_STAMP(4 + (w >> 3), j, w & 7);
         if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
     }
-    if (lane == 0 && w == 0) FTL_STAMP(3, 0, 2);
 
     // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R/l - (mu - c) O, lse = ln2 (m + log2 l)
     if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, FWD_WAIT_LIMIT_NS);
@@ -367,7 +324,6 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const uint32_t bar0 = ptx::smem_u32(misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48 * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 48 * 8 + 16);
-    const uint32_t turn_addr = bar0 + 48 * 8 + 32;  // turn counter of the two MMA issuers
     float* xmax = reinterpret_cast<float*>(misc + 48 * 8 + 64);
     float* xslow = xmax + C::XMAX_FLOATS;
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
@@ -380,7 +336,6 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        *reinterpret_cast<volatile uint32_t*>(misc + 48 * 8 + 32) = 0u;
         for (int s = 0; s < SE; ++s) { ptx::mbar_init(bar(C::B_EFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_EEMPTY + s), 1); }
         for (int s = 0; s < SL; ++s) { ptx::mbar_init(bar(C::B_LFULL + s), C::FULL_COUNT); ptx::mbar_init(bar(C::B_LEMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
@@ -416,7 +371,6 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 0) FTL_STAMP(3, 0, 0);
 
     // shared-memory address of tile `t` (0 = K, 1 = tK in the E ring; 2 = V, 3 = tV in the L ring) of iteration j
     auto tile_addr = [&](int t, int j) -> uint32_t {
@@ -470,27 +424,22 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             if (lane == 0) ptx::mbar_arrive(bar(b_full + (T - 1) % S));
         }
         if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
-    } else if (warp == 1 || warp == 3) {
-        // ------------------------------------------------------------------ MMA issuers, warps 1 and 3, on two
-        // schedulers.  Each whole warp runs its loop in converged control flow; one elected lane issues (see
-        // mma_ts_elect).  An issuing thread is held at the rate of the tensor pipe while its MMAs are queued,
-        // and the waits between two steps cost it several hundred clocks next to the element-wise warps of its
-        // scheduler, so the tiles alternate: warp 1 takes the even ones (score buffer 0), warp 3 the odd ones.
-        // A tile's value MMAs and the score MMAs of the tile after next, which overwrite their operands, come
-        // from one thread, so the pipe orders them.  A turn counter passes from batch to batch: it keeps the
-        // accumulation in tile order, and two batches queued at once would share the pipe MMA by MMA and
-        // finish late and together.
-        const int wsel = warp >> 1;
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ score MMAs (warp 1) and value MMAs
+        // (warp 3), on two schedulers: an MMA costs 7 to 14 issue slots of its scheduler, which the element-wise
+        // warps of that quadrant also need.  Each whole warp runs its loop in converged control flow; one
+        // elected lane issues (see mma_ts_elect).
         constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
-        constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
         const uint32_t aq = tb + C::COL_Q, atq = tb + C::COL_TQ;
-        const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
-        auto issue_scores = [&](int j) -> bool {
+        bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, FWD_WAIT_LIMIT_NS);
+        for (int j = 0; ok && j < T; ++j) {
             const int b = j & 1;
-            if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
+            ok = ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            // the score buffer is free once the value MMAs of tile j-2 have read their operands out of it
+            if (ok && j >= 2) ok = ptx::mbar_wait_warp(bar(C::B_OUTDONE + b), ((j - 2) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (!ok) break;
             ptx::tc_fence_after_sync();
-            if (lane == 0) FTL_STAMP(0, j, 0);
             const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
             const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
@@ -512,17 +461,18 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             }
             ptx::mma_commit_elect(bar(C::B_SFULL + 2 + b));
             ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
-            if (lane == 0) FTL_STAMP(0, j, 1);
-            return true;
-        };
-        auto issue_values = [&](int j) -> bool {
+        }
+    } else if (warp == 3) {
+        constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+        bool ok = true;
+        for (int j = 0; ok && j < T; ++j) {
             const int b = j & 1;
-            if (lane == 0) FTL_STAMP(0, j, 2);
-            if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
-            if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
-            if (!ptx::turn_wait_warp(turn_addr, (uint32_t)j, abort_flag, FWD_WAIT_LIMIT_NS)) return false;
+            ok = ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (!ok) break;
             ptx::tc_fence_after_sync();
-            if (lane == 0) FTL_STAMP(0, j, 3);
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
             const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
@@ -538,17 +488,6 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
             ptx::mma_commit_elect(bar(C::B_OUTDONE + b));
             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
-            if (lane == 0) FTL_STAMP(0, j, 4);
-            return true;
-        };
-        bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, FWD_WAIT_LIMIT_NS);
-        if (ok && wsel < T) ok = issue_scores(wsel);
-        for (int j = wsel; ok && j < T; j += 2) {
-            ok = issue_values(j);
-            if (ok && j + 2 < T) ok = issue_scores(j + 2);
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)j + 1u);
         }
     } else if (warp >= 4) {
         fwd_elementwise<DP>(p, tmem_base, bar0, abort_flag, xmax, xslow, warp - 4, lane, bh, row0, T);
@@ -557,7 +496,6 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // ---------------------------------------------------------------------- teardown
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0) FTL_STAMP(3, 0, 1);
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, 512);
