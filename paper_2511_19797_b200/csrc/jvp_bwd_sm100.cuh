@@ -175,15 +175,30 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     const size_t grow = (size_t)bh * p.N + row0 + row;
 
     // ---- owner rows of X0 and X1 -> bf16 operands in tensor memory (k-step kk at 8 packed columns)
-    for (int ch = slot; ch < 2 * KS; ch += 4) {
-        const bool second = ch >= KS;
-        const int kk = second ? ch - KS : ch;
-        const __nv_bfloat16* src = p.own[second ? 1 : 0] + grow * p.d + 16 * kk;
-        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
-        if (row_valid && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
-        if (row_valid && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
-        const uint32_t r[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        ptx::tmem_st8(lane_addr + (second ? C::COL_X1 : C::COL_X0) + 8 * kk, r);
+    // all of this warp's loads first, then the stores: one global-memory latency instead of one per chunk
+    {
+        constexpr int NCH = (2 * KS + 3) / 4;  // chunks of 16 columns per warp, at most
+        uint4 v[NCH][2];
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int ch = slot + 4 * i;
+            const bool second = ch >= KS;
+            const int kk = second ? ch - KS : ch;
+            const __nv_bfloat16* src = p.own[second ? 1 : 0] + grow * p.d + 16 * kk;
+            v[i][0] = v[i][1] = make_uint4(0, 0, 0, 0);
+            if (ch < 2 * KS && row_valid && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
+            if (ch < 2 * KS && row_valid && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
+        }
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int ch = slot + 4 * i;
+            if (ch < 2 * KS) {
+                const bool second = ch >= KS;
+                const int kk = second ? ch - KS : ch;
+                const uint32_t r[8] = {v[i][0].x, v[i][0].y, v[i][0].z, v[i][0].w, v[i][1].x, v[i][1].y, v[i][1].z, v[i][1].w};
+                ptx::tmem_st8(lane_addr + (second ? C::COL_X1 : C::COL_X0) + 8 * kk, r);
+            }
+        }
     }
     ptx::tmem_wait_st();
     ptx::tc_fence_before_sync();

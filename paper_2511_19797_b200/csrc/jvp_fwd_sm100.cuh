@@ -114,15 +114,27 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
     const size_t grow = (size_t)bh * p.N + row0 + row;
 
     // ---- Q and tQ rows -> bf16 operands in tensor memory (k-step kk at 8 packed columns)
-    for (int ch = sl; ch < 2 * KS; ch += 4) {
-        const bool is_t = ch >= KS;
-        const int kk = is_t ? ch - KS : ch;
-        const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow * p.d + 16 * kk;
-        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
-        if (row_valid && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
-        if (row_valid && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
-        const uint32_t r[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        ptx::tmem_st8(lane_addr + (is_t ? C::COL_TQ : C::COL_Q) + 8 * kk, r);
+    {
+        // the loads of the next chunk are in flight while this one is stored
+        auto load = [&](int ch, uint4& v0, uint4& v1) {
+            const bool is_t = ch >= KS;
+            const int kk = is_t ? ch - KS : ch;
+            const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow * p.d + 16 * kk;
+            v0 = v1 = make_uint4(0, 0, 0, 0);
+            if (ch < 2 * KS && row_valid && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
+            if (ch < 2 * KS && row_valid && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
+        };
+        uint4 v0, v1, n0, n1;
+        load(sl, v0, v1);
+        for (int ch = sl; ch < 2 * KS; ch += 4) {
+            load(ch + 4, n0, n1);
+            const bool is_t = ch >= KS;
+            const int kk = is_t ? ch - KS : ch;
+            const uint32_t r[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+            ptx::tmem_st8(lane_addr + (is_t ? C::COL_TQ : C::COL_Q) + 8 * kk, r);
+            v0 = n0;
+            v1 = n1;
+        }
     }
     ptx::tmem_wait_st();
     ptx::tc_fence_before_sync();
@@ -209,19 +221,23 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
                 // accumulators must be at rest: the value MMAs of tile j-1 have completed
                 if (!ptx::mbar_wait(bar(C::B_OUTDONE + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
-                for (int ch = sl; ch < KS; ch += 4) {
-                    uint32_t o[16], r[16];
-                    ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
-                    ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, r);
-                    ptx::tmem_wait_ld();
+                // eight columns at a time: this rare path must not set the register peak of the loop
+                for (int ch = 2 * sl; ch < 2 * KS; ch += 8) {
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t o[8], r[8];
+                        ptx::tmem_ld8(lane_addr + C::COL_ACC0 + 8 * (ch + h), o);
+                        ptx::tmem_ld8(lane_addr + C::COL_ACC1 + 8 * (ch + h), r);
+                        ptx::tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float ov = __uint_as_float(o[c]);
-                        r[c] = __float_as_uint(scale * fmaf(fix, ov, __uint_as_float(r[c])));
-                        o[c] = __float_as_uint(scale * ov);
+                        for (int c = 0; c < 8; ++c) {
+                            const float ov = __uint_as_float(o[c]);
+                            r[c] = __float_as_uint(scale * fmaf(fix, ov, __uint_as_float(r[c])));
+                            o[c] = __float_as_uint(scale * ov);
+                        }
+                        ptx::tmem_st8(lane_addr + C::COL_ACC0 + 8 * (ch + h), o);
+                        ptx::tmem_st8(lane_addr + C::COL_ACC1 + 8 * (ch + h), r);
                     }
-                    ptx::tmem_st16(lane_addr + C::COL_ACC0 + 16 * ch, o);
-                    ptx::tmem_st16(lane_addr + C::COL_ACC1 + 16 * ch, r);
                 }
             }
         }
