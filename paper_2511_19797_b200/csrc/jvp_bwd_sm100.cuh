@@ -375,6 +375,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                const BwdParams p) {
     using C = BwdCfg<MODE, DP>;
     constexpr int BC = C::BC, KS = C::KS, NA = C::NA, SE = C::SE, SL = C::SL, NPAIR = C::NPAIR;
+    // the next backward pass in the stream, if launched as a programmatic dependent, may start as SMs free up
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (*reinterpret_cast<volatile int*>(p.status) != 0) return;  // an earlier kernel timed out
 
     extern __shared__ uint8_t smem_raw[];

@@ -241,7 +241,25 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
         return TVM_ATTN_CUDA_ERROR;
     const long long grid = s.BH * ((s.N + BWD_ROWS - 1) / BWD_ROWS);
     g_prof.before(st);
-    kern<<<(unsigned)grid, BWD_THREADS, C::SMEM_BYTES, st>>>(ms[0], ms[1], ms[2], ms[3], mo[0], mo[1], prm);
+    {
+        // DK and DQ read nothing that the pass before them writes (DV, DK and DQ all depend on the row-sums
+        // pre-pass only, which has completed before DV starts), so their CTAs may fill the SMs that the last,
+        // partial wave of the pass before leaves idle: programmatic dependent launch, with every CTA of these
+        // kernels releasing its dependents at once and none waiting for its primary.  Not while per-kernel
+        // events are being recorded: they would time overlapping kernels.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(BWD_THREADS);
+        cfg.dynamicSmemBytes = C::SMEM_BYTES;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = (MODE != BWD_DV && !g_prof.enabled) ? 1 : 0;
+        if (cudaLaunchKernelEx(&cfg, kern, ms[0], ms[1], ms[2], ms[3], mo[0], mo[1], prm) != cudaSuccess)
+            return cuda_status(cudaGetLastError());
+    }
     g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
