@@ -7,7 +7,12 @@
 //     O~ += P~ V,  R += (P~ (T - c)) V + P~ tV    (three GEMMs per key tile)
 //     O = O~/l,  tO = R/l - (mu - c) O,  lse = ln2 (m + log2 l),  mu = c + sum(P~ (T - c))/l
 //
-// A CTA owns 128 query rows of one head and streams the keys in tiles of 64.
+// A work item is 128 query rows of one head, against which the head's keys stream in tiles of 64.  The
+// grid has one CTA per SM (a CTA needs the whole tensor memory of one); the items go round-robin over
+// the CTAs.  The shared-memory rings, the score buffers and all barrier phases run on through the items,
+// so the loads, the operand staging and the first score MMAs of an item are under way while the
+// element-wise warps still normalise and store the item before.  (One CTA per item spent a quarter of
+// its life on set-up and epilogue at N = 1024.)
 //
 // What is where
 //   * Q and tQ of the CTA's rows are written once into tensor memory as bf16 operands, so the three
@@ -103,26 +108,29 @@ struct FwdCfg {
 template <int DP>
 __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tmem_base, uint32_t bar0,
                                                 volatile int* abort_flag, float* xmax, float* xslow, int w, int lane,
-                                                int bh, int row0, int T) {
+                                                int items, int row_tiles, int T) {
     using C = FwdCfg<DP>;
     constexpr int BC = FWD_BC, KS = C::KS;
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
     const int q = w & 3, sl = w >> 2;
     const int row = q * 32 + lane;  // query row inside the CTA tile
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-    const bool row_valid = row0 + row < p.N;
-    const size_t grow = (size_t)bh * p.N + row0 + row;
 
-    // ---- Q and tQ rows -> bf16 operands in tensor memory (k-step kk at 8 packed columns)
-    {
+    // ---- Q and tQ rows of an item -> bf16 operands in tensor memory (k-step kk at 8 packed columns).  Called
+    // once the warp has seen the last scores of the item before: no MMA reads the old operands any more.
+    auto stage_q = [&](int item) {
+        const int bh_ = item / row_tiles;
+        const int row0_ = (item - bh_ * row_tiles) * FWD_ROWS;
+        const bool valid_ = row0_ + row < p.N;
+        const size_t grow_ = (size_t)bh_ * p.N + row0_ + row;
         // the loads of the next chunk are in flight while this one is stored
         auto load = [&](int ch, uint4& v0, uint4& v1) {
             const bool is_t = ch >= KS;
             const int kk = is_t ? ch - KS : ch;
-            const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow * p.d + 16 * kk;
+            const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow_ * p.d + 16 * kk;
             v0 = v1 = make_uint4(0, 0, 0, 0);
-            if (ch < 2 * KS && row_valid && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
-            if (ch < 2 * KS && row_valid && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
+            if (ch < 2 * KS && valid_ && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
+            if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
         };
         uint4 v0, v1, n0, n1;
         load(sl, v0, v1);
@@ -135,23 +143,31 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             v0 = n0;
             v1 = n1;
         }
-    }
-    ptx::tmem_wait_st();
-    ptx::tc_fence_before_sync();
-    __syncwarp();
-    if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+    };
 
-    float m_ref = -CUDART_INF_F, cen = 0.f;
-    uint64_t l2 = 0ull, mt2 = 0ull;  // two partial sums each of P~ and of P~(T - c) over this warp's slices
-    int n_slow = 0;                  // exchanges done on B_XSLOW
+    int n_slow = 0;  // exchanges done on B_XSLOW
     bool ok = true;
     const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
     float2* xs2 = reinterpret_cast<float2*>(xslow);
+    int g = 0, it = 0;  // tiles and items done by this CTA
+    if ((int)blockIdx.x < items) stage_q(blockIdx.x);
 
-    for (int j = 0; j < T; ++j) {
-        const int b = j & 1;
+    for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
+    const int bh = item / row_tiles;
+    const int row0 = (item - bh * row_tiles) * FWD_ROWS;
+    const bool row_valid = row0 + row < p.N;
+    const size_t grow = (size_t)bh * p.N + row0 + row;
+    float m_ref = -CUDART_INF_F, cen = 0.f;
+    uint64_t l2 = 0ull, mt2 = 0ull;  // two partial sums each of P~ and of P~(T - c) over this warp's slices
+
+    for (int j = 0; j < T; ++j, ++g) {
+        const int b = g & 1;
         // S is complete before Sd: the row maxima are found and exchanged while the Sd MMAs still run
-        if (!ptx::mbar_wait(bar(C::B_SFULL + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        if (!ptx::mbar_wait(bar(C::B_SFULL + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS;
         uint32_t s[16], ts[16];
@@ -168,14 +184,14 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
 #pragma unroll
         for (int c = 3; c < 15; c += 2) mx = ptx::max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
         mx = fmaxf(mx, __uint_as_float(s[15]));
-        float* xm = xmax + (j & 1) * 512;
+        float* xm = xmax + (g & 1) * 512;
         xm[row * 4 + sl] = mx;
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(bar(C::B_XMAX + q));
-        if (!ptx::mbar_wait(bar(C::B_SFULL + 2 + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        if (!ptx::mbar_wait(bar(C::B_SFULL + 2 + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
-        if (!ptx::mbar_wait(bar(C::B_XMAX + q), j & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        if (!ptx::mbar_wait(bar(C::B_XMAX + q), g & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
         const float4 o4 = *reinterpret_cast<const float4*>(xm + row * 4);
         const float mrow = fmaxf(ptx::max3(o4.x, o4.y, o4.z), o4.w) * p.c2;  // tile maximum of the row, log2 units
         ptx::tmem_wait_ld();
@@ -219,7 +235,7 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             }
             if (j > 0) {
                 // accumulators must be at rest: the value MMAs of tile j-1 have completed
-                if (!ptx::mbar_wait(bar(C::B_OUTDONE + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                if (!ptx::mbar_wait(bar(C::B_OUTDONE + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
                 // eight columns at a time: this rare path must not set the register peak of the loop
                 for (int ch = 2 * sl; ch < 2 * KS; ch += 8) {
@@ -269,8 +285,11 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
         if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
     }
 
+    if (!ok) break;
+    // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
+    if (item + (int)gridDim.x < items) stage_q(item + gridDim.x);
     // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R/l - (mu - c) O, lse = ln2 (m + log2 l)
-    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, FWD_WAIT_LIMIT_NS);
+    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
     if (ok) {
         ptx::tc_fence_after_sync();
         float l0, l1, t0, t1;
@@ -280,6 +299,7 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
         ok = ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+        ++n_slow;
     }
     if (ok) {
         float l = 0.f, mt = 0.f;
@@ -321,6 +341,7 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             p.mu[grow] = cen + mun;
         }
     }
+    }
 }
 
 template <int DP>
@@ -345,10 +366,13 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Work items (a head and 128 of its query rows) go round-robin over the CTAs of a grid that has one
+    // CTA per SM.  The rings, the score buffers and every barrier phase run on through the items (tile
+    // counter g), so the loads and the first score MMAs of an item are under way while the element-wise
+    // warps still write out the item before.
     const int row_tiles = (p.N + FWD_ROWS - 1) / FWD_ROWS;
-    const int bh = blockIdx.x / row_tiles;
-    const int row0 = (blockIdx.x - bh * row_tiles) * FWD_ROWS;
-    const int T = (p.N + BC - 1) / BC;  // key tiles
+    const int items = p.BH * row_tiles;
+    const int T = (p.N + BC - 1) / BC;  // key tiles per item
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -400,46 +424,84 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // end of a 144-byte row would read the next row's bytes from L2 only to replace them by zeros,
         // which nearly doubled the L2 traffic), and signal them one tile later so that two tiles of copies
         // are in flight.
+        // Kept to a few dozen instructions per tile: everything that does not depend on the tile (lane's
+        // row, chunk positions, source pointers) is set up before the loops.
         const int ring = warp >> 1;
         const int S = ring == 0 ? SE : SL;
         const int b_full = ring == 0 ? C::B_EFULL : C::B_LFULL, b_empty = ring == 0 ? C::B_EEMPTY : C::B_LEMPTY;
-        const CUtensorMap* maps[2] = {ring == 0 ? &tm_k : &tm_v, ring == 0 ? &tm_tk : &tm_tv};
-        const __nv_bfloat16* srcs[2] = {ring == 0 ? p.K : p.V, ring == 0 ? p.tK : p.tV};
-        const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
+        constexpr uint32_t TB = C::ST_BYTES;
+        constexpr int KT = NA == 2 ? (DP - 64) / 8 : 1;  // 16-byte chunks per row behind column 64, at most
+        const CUtensorMap* map0 = ring == 0 ? &tm_k : &tm_v;
+        const CUtensorMap* map1 = ring == 0 ? &tm_tk : &tm_tv;
+        const uint32_t ring_base = ring == 0 ? e_base : l_base;
+        const __nv_bfloat16* base0 = ring == 0 ? p.K : p.V;
+        const __nv_bfloat16* base1 = ring == 0 ? p.tK : p.tV;
+        [[maybe_unused]] const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
+        [[maybe_unused]] const int d32 = 32 * p.d;
+        [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
+        [[maybe_unused]] const uint32_t dst_lane = BC * 128 + lane * 128;
+        [[maybe_unused]] const uint32_t sw = lane & 7;
         bool ok = true;
-        for (int j = 0; j < T; ++j) {
-            const int s = j % S, ph = (j / S) & 1;
-            ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            if (!ok) break;
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
-                for (int t = 0; t < 2; ++t) ptx::tma_load_3d(tile_addr(2 * ring + t, j), maps[t], bar(b_full + s), 0, j * BC, bh);
-            }
-            if constexpr (NA == 2) {
-                for (int i = lane; i < 2 * BC * ntail; i += 32) {
-                    const int t = i / (BC * ntail), rem = i - t * (BC * ntail);
-                    const int r = rem / ntail, k = rem - r * ntail;
-                    const int grow = j * BC + r;
-                    const bool v = grow < p.N;
-                    const __nv_bfloat16* src = srcs[t] + ((size_t)bh * p.N + (v ? grow : 0)) * p.d + 64 + 8 * k;
-                    ptx::cp_async_16(tile_addr(2 * ring + t, j) + BC * 128 + r * 128 + ((k ^ (r & 7)) << 4), src, v ? 16u : 0u);
+        int s = 0, ph = 0, pend_s = -1;
+        for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+            const int bh = item / row_tiles;
+            [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;
+            [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;
+            [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
+            for (int j = 0; j < T; ++j) {
+                if constexpr (NA == 2) {
+                    if (pend_s >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
+                        ptx::cp_async_wait<0>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                        pend_s = -1;
+                    }
                 }
-                ptx::cp_async_commit();
-                if (j > 0) {
-                    ptx::cp_async_wait<1>();
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(b_full + (j - 1) % S));
+                ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, FWD_WAIT_LIMIT_NS);
+                if (!ok) break;
+                const uint32_t stage = ring_base + s * 2 * TB;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
+                    ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
+                    ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
                 }
+                if constexpr (NA == 2) {
+                    const int rows_left = p.N - j * BC;
+#pragma unroll
+                    for (int k = 0; k < KT; ++k) {
+                        if (k < ntail) {
+#pragma unroll
+                            for (int rp = 0; rp < BC / 32; ++rp) {
+                                const bool v = lane + 32 * rp < rows_left;
+                                const uint32_t dst = stage + dst_lane + rp * 32 * 128 + ((k ^ sw) << 4);
+                                ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
+                                ptx::cp_async_16(dst + TB, v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                            }
+                        }
+                    }
+                    ptx::cp_async_commit();
+                    if (pend_s >= 0) {
+                        ptx::cp_async_wait<1>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                    }
+                    pend_s = s;
+                    src0 += tile_elems;
+                    src1 += tile_elems;
+                }
+                if (++s == S) { s = 0; ph ^= 1; }
             }
         }
-        if (NA == 2 && ok) {
-            ptx::cp_async_wait<0>();
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(b_full + (T - 1) % S));
+        if (NA == 2) {
+            ptx::cp_async_wait<0>();  // nothing of ours stays in flight
+            if (ok && pend_s >= 0) {
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+            }
         }
-        if (NA == 2 && !ok) ptx::cp_async_wait<0>();  // nothing of ours stays in flight
     } else if (warp == 1) {
         // ------------------------------------------------------------------ score MMAs (warp 1) and value MMAs
         // (warp 3), on two schedulers: an MMA costs 7 to 14 issue slots of its scheduler, which the element-wise
@@ -448,16 +510,21 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(128, BC, 0, 0);
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
         const uint32_t aq = tb + C::COL_Q, atq = tb + C::COL_TQ;
-        bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, FWD_WAIT_LIMIT_NS);
-        for (int j = 0; ok && j < T; ++j) {
-            const int b = j & 1;
-            ok = ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            // the score buffer is free once the value MMAs of tile j-2 have read their operands out of it
-            if (ok && j >= 2) ok = ptx::mbar_wait_warp(bar(C::B_OUTDONE + b), ((j - 2) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+        bool ok = true;
+        int g = 0, it = 0;
+        for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
+        // Q, tQ of this item are in tensor memory (the element-wise warps stage them as soon as they have
+        // seen the last scores of the item before)
+        ok = ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+        for (int j = 0; ok && j < T; ++j, ++g) {
+            const int b = g & 1;
+            ok = ptx::mbar_wait_warp(bar(C::B_EFULL + g % SE), (g / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            // the score buffer is free once the value MMAs of tile g-2 have read their operands out of it
+            if (ok && g >= 2) ok = ptx::mbar_wait_warp(bar(C::B_OUTDONE + b), ((g - 2) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, j), 16, 1024);
-            const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, j), 16, 1024);
+            const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, g), 16, 1024);
+            const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, g), 16, 1024);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk) {  // S = Q K^T
@@ -476,23 +543,29 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
             }
             ptx::mma_commit_elect(bar(C::B_SFULL + 2 + b));
-            ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+            ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
+        }
         }
     } else if (warp == 3) {
         constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
         const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
         bool ok = true;
-        for (int j = 0; ok && j < T; ++j) {
-            const int b = j & 1;
-            ok = ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+        int g = 0;
+        for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+        // The first tile of an item overwrites the accumulators (accumulate = 0): every element-wise warp
+        // reads them out for the item before (its epilogue) before it turns to this tile, whose operands
+        // the wait below is for.
+        for (int j = 0; ok && j < T; ++j, ++g) {
+            const int b = g & 1;
+            ok = ptx::mbar_wait_warp(bar(C::B_LFULL + g % SL), (g / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
-            const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
-            const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+            const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);
+            const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
 #pragma unroll
             for (int u = 0; u < BC / 16; ++u) {
                 const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
@@ -501,12 +574,13 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 ptx::mma_ts_elect(acc1, a1 + 16 * u, vd + off, idesc_o, acc);   // R  += P~(T-c) V
                 ptx::mma_ts_elect(acc1, a0 + 16 * u, tvd + off, idesc_o, 1u);   // R  += P~ tV
             }
-            ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+            ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
             ptx::mma_commit_elect(bar(C::B_OUTDONE + b));
             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
         }
+        }
     } else if (warp >= 4) {
-        fwd_elementwise<DP>(p, tmem_base, bar0, abort_flag, xmax, xslow, warp - 4, lane, bh, row0, T);
+        fwd_elementwise<DP>(p, tmem_base, bar0, abort_flag, xmax, xslow, warp - 4, lane, items, row_tiles, T);
     }
 
     // ---------------------------------------------------------------------- teardown

@@ -213,7 +213,13 @@ static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams
     auto kern = jvp_fwd_kernel<DP>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
         return TVM_ATTN_CUDA_ERROR;
-    const long long grid = s.BH * ((s.N + FWD_ROWS - 1) / FWD_ROWS);
+    // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
+    // items go round-robin over them
+    const long long items = s.BH * ((s.N + FWD_ROWS - 1) / FWD_ROWS);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return TVM_ATTN_CUDA_ERROR;
+    const long long grid = items < sms ? items : sms;
     g_prof.before(st);
     kern<<<(unsigned)grid, FWD_THREADS, C::SMEM_BYTES, st>>>(m[0], m[1], m[2], m[3], prm);
     g_prof.after(st);
