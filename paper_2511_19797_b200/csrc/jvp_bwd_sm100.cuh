@@ -10,7 +10,10 @@
 // with P = 2^(c2 S - lse2), Nn = alpha Sd - mu, W = P (D - Sigma1), dA = P (X - c) + W Nn, and
 //   acc0 += A0 B0,  acc1 += A1 B0 + A0 B1      (B0, B1 = Hc, G | Q, tQ | K, tK).
 //
-// A CTA owns 128 owner rows of one head and streams the other side in tiles of BC = 64 rows.
+// A work item is 128 owner rows of one head, against which the other side streams in tiles of BC = 64
+// rows.  The grid has one CTA per SM (a CTA needs the whole tensor memory of one); the items go round-robin
+// over the CTAs, and the rings, the score buffers and all barrier phases run on through the items, so the
+// loads, the operand staging and the first score MMAs of an item overlap the epilogue of the item before.
 //
 // What is where
 //   * The owner operands of the first score pair (K, tK or Q, tQ) are written once into tensor memory
@@ -123,7 +126,9 @@ struct BwdCfg {
     static constexpr int B_FINAL = B_PREADY + 2;
     static constexpr int B_QREADY = B_FINAL + 1;
     static constexpr int B_OWNER = B_QREADY + 1;
-    static constexpr int NBARS = B_OWNER + 1;
+    static constexpr int B_ACCFREE = B_OWNER + 1;  // the element-wise warps have read the accumulators of an item
+    static constexpr int B_OWNFREE = B_ACCFREE + 1;  // the MMAs that read the shared-memory owner tiles of an item are done
+    static constexpr int NBARS = B_OWNFREE + 1;
     static_assert(NBARS <= 48, "barrier table too small");
     static constexpr int STATS_FLOATS = SL * 4 * 64;
     static constexpr int MISC_BYTES = 48 * 8 + 64 + STATS_FLOATS * 4;
@@ -157,8 +162,8 @@ __device__ __forceinline__ void bwd_element(const BwdParams& p, float s, float t
 // Element-wise warps of the backward passes: `w` in 0..15.
 template <int MODE, int DP>
 __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tmem_base, uint32_t bar0,
-                                                volatile int* abort_flag, const float* stats, int w, int lane, int bh,
-                                                int row0, int T) {
+                                                volatile int* abort_flag, const float* stats, int w, int lane, int items,
+                                                int row_tiles, int T) {
     using C = BwdCfg<MODE, DP>;
     constexpr int BC = C::BC, KS = C::KS, NPAIR = C::NPAIR;
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
@@ -171,12 +176,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     const int sl = NPAIR == 1 ? 2 * (slot & 1) : slot;  // first (or only) slice of this warp
     const int row = q * 32 + lane;  // owner row inside the CTA tile
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-    const bool row_valid = row0 + row < p.N;
-    const size_t grow = (size_t)bh * p.N + row0 + row;
 
-    // ---- owner rows of X0 and X1 -> bf16 operands in tensor memory (k-step kk at 8 packed columns)
-    // all of this warp's loads first, then the stores: one global-memory latency instead of one per chunk
-    {
+    // ---- owner rows of X0 and X1 of an item -> bf16 operands in tensor memory (k-step kk at 8 packed
+    // columns); all of this warp's loads first, then the stores: one global-memory latency instead of one
+    // per chunk.  Called once no MMA reads the operands of the item before any more.
+    auto stage_x = [&](int item) {
+        const int bh_ = item / row_tiles;
+        const int row0_ = (item - bh_ * row_tiles) * BWD_ROWS;
+        const bool valid_ = row0_ + row < p.N;
+        const size_t grow_ = (size_t)bh_ * p.N + row0_ + row;
         constexpr int NCH = (2 * KS + 3) / 4;  // chunks of 16 columns per warp, at most
         uint4 v[NCH][2];
 #pragma unroll
@@ -184,10 +192,10 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             const int ch = slot + 4 * i;
             const bool second = ch >= KS;
             const int kk = second ? ch - KS : ch;
-            const __nv_bfloat16* src = p.own[second ? 1 : 0] + grow * p.d + 16 * kk;
+            const __nv_bfloat16* src = p.own[second ? 1 : 0] + grow_ * p.d + 16 * kk;
             v[i][0] = v[i][1] = make_uint4(0, 0, 0, 0);
-            if (ch < 2 * KS && row_valid && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
-            if (ch < 2 * KS && row_valid && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
+            if (ch < 2 * KS && valid_ && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
+            if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
         }
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
@@ -199,12 +207,21 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 ptx::tmem_st8(lane_addr + (second ? C::COL_X1 : C::COL_X0) + 8 * kk, r);
             }
         }
-    }
-    ptx::tmem_wait_st();
-    ptx::tc_fence_before_sync();
-    __syncwarp();
-    if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+    };
 
+    bool ok = true;
+    int it = 0;  // items done by this CTA
+    if ((int)blockIdx.x < items) stage_x(blockIdx.x);
+    for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
+    const int g0 = it * T;  // tiles this CTA has streamed before this item: rings and barrier phases run on
+    const int bh = item / row_tiles;
+    const int row0 = (item - bh * row_tiles) * BWD_ROWS;
+    const bool row_valid = row0 + row < p.N;
+    const size_t grow = (size_t)bh * p.N + row0 + row;
     float r_lse2 = CUDART_INF_F, r_mu = 0.f, r_s1 = 0.f, r_cv = 0.f;  // per-row statistics (DQ)
     if (MODE == BWD_DQ && row_valid) {
         r_lse2 = p.lse2[grow];
@@ -212,15 +229,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         r_s1 = p.sig1[grow];
         r_cv = p.cvec[grow];
     }
-    bool ok = true;
-    for (int j = par; j < T; j += jstep) {
-        const int b = NPAIR == 1 ? (j & 1) : 0, sph = NPAIR == 1 ? (j >> 1) & 1 : (j & 1);
+    for (int j = NPAIR == 1 ? ((par ^ g0) & 1) : 0; j < T; j += jstep) {
+        const int g = g0 + j;
+        const int b = NPAIR == 1 ? (g & 1) : 0, sph = NPAIR == 1 ? (g >> 1) & 1 : (g & 1);
         if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
         // the statistics of the tile's queries arrive with its L stage, which is not released before the
         // output MMAs of this tile, hence not before every warp is through with them
-        const float* st = stats + (j % C::SL) * 4 * 64 + 16 * sl;
+        const float* st = stats + (g % C::SL) * 4 * 64 + 16 * sl;
         if (C::TRANSPOSED)
-            if (!ptx::mbar_wait(bar(C::B_LFULL + j % C::SL), (j / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            if (!ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 0);
         const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
@@ -307,7 +324,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             }
             // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
             if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 2);
-            if (!ptx::mbar_wait(bar(C::B_SFULL + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            if (!ptx::mbar_wait(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 3);
             uint32_t s3[16], s4[16];
@@ -339,7 +356,18 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         if (lane == 0) BTL_STAMP(4 + (w >> 3), j, w & 7);
         if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
     }
-    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), 0, abort_flag, BWD_WAIT_LIMIT_NS);
+    if (!ok) break;
+    // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
+    if (item + (int)gridDim.x < items) {
+        if (NPAIR == 1) {
+            // DV: this warp has seen only the scores of its own tiles; those of the item's last tile, which
+            // may belong to the other eight warps, must be complete too before the operands change
+            const int gl = g0 + T - 1;
+            if (!ptx::mbar_wait(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+        }
+        stage_x(item + gridDim.x);
+    }
+    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
     if (ok) {
         ptx::tc_fence_after_sync();
         __nv_bfloat16* p0 = p.out0 + grow * p.d;
@@ -364,6 +392,11 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 }
             }
         }
+        // the accumulators may be overwritten by the first output MMAs of the next item
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_ACCFREE));
+    }
     }
 }
 
@@ -393,10 +426,13 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Work items (a head and 128 of its owner rows) go round-robin over the CTAs of a grid that has one CTA
+    // per SM.  The rings, the score buffers and every barrier phase run on through the items (tile counter
+    // g), so the loads, the operand staging and the first score MMAs of an item are under way while the
+    // element-wise warps still write out the item before.
     const int row_tiles = (p.N + BWD_ROWS - 1) / BWD_ROWS;
-    const int bh = blockIdx.x / row_tiles;
-    const int row0 = (blockIdx.x - bh * row_tiles) * BWD_ROWS;
-    const int T = (p.N + BC - 1) / BC;  // stream tiles
+    const int items = p.BH * row_tiles;
+    const int T = (p.N + BC - 1) / BC;  // stream tiles per item
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -410,6 +446,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         ptx::mbar_init(bar(C::B_FINAL), 1);
         ptx::mbar_init(bar(C::B_QREADY), 16);
         ptx::mbar_init(bar(C::B_OWNER), C::FULL_COUNT);
+        ptx::mbar_init(bar(C::B_ACCFREE), 16);
+        ptx::mbar_init(bar(C::B_OWNFREE), 1);
         ptx::fence_mbar_init();
     }
     if (NA == 2) {
@@ -459,7 +497,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         // does not depend on the tile (lane's row, chunk positions, source pointers) is set up before it.
         constexpr int KT = NA == 2 ? (DP - 64) / 8 : 1;  // 16-byte chunks per row behind column 64, at most
         const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
-        const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
         const int d32 = 32 * p.d;                                      // 32 rows further down, in elements
         bool owner_pend = false;  // owner-tile copies issued (warp 0) and not signalled yet
         auto produce = [&](auto ring_tag) -> void {
@@ -475,8 +512,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const uint32_t ring_base = ring == 0 ? e_base : l_base;
             const __nv_bfloat16* base0 = p.strm[2 * ring];
             const __nv_bfloat16* base1 = p.strm[2 * ring + 1];
-            [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
-            [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
             [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
             // Destination of chunk 0 of row `lane` behind the 64-column atom: the E ring keeps compact
             // 16-byte-per-row blocks (K-major operands only), the L ring a second 128-byte-swizzled atom.
@@ -485,11 +520,60 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // statistics: 16-byte chunks when the rows of the (B, H, N) arrays are 16-byte aligned, else floats
             const bool st16 = (p.N & 3) == 0;
             [[maybe_unused]] const uint32_t st_base = ptx::smem_u32(stats);
+            bool ok = true;
+            int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
+            int it = 0;
+            for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
+            const int bh = item / row_tiles;
+            [[maybe_unused]] const int row0 = (item - bh * row_tiles) * BWD_ROWS;
+            [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
+            [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
+            [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
             [[maybe_unused]] const size_t srow = (size_t)bh * p.N;
             [[maybe_unused]] const float* st_src0 = (lane < 16 ? p.lse2 : p.mu) + srow + 4 * (lane & 15);
             [[maybe_unused]] const float* st_src1 = NST == 4 ? (lane < 16 ? p.sig1 : p.cvec) + srow + 4 * (lane & 15) : nullptr;
-            bool ok = true;
-            int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
+            if constexpr (ring == 0 && NPAIR == 2) {
+                // The shared-memory owner tiles of this item, once the MMAs that read those of the item before
+                // are done.  Their copied columns are signalled with the first tile's: nothing needs them earlier.
+                if (it > 0) {
+                    if constexpr (HAS_CP) {
+                        // the MMAs waited for below need the last tile of the item before: signal its copies first
+                        if (pend_s >= 0) {
+                            ptx::cp_async_wait<0>();
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                            pend_s = -1;
+                        }
+                    }
+                    ok = ptx::mbar_wait_warp(bar(C::B_OWNFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    if (!ok) break;
+                }
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
+                    ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
+                    ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
+                }
+                if constexpr (NA == 2) {
+                    const __nv_bfloat16* o2 = p.own[2] + lane_row + (size_t)row0 * p.d;
+                    const __nv_bfloat16* o3 = p.own[3] + lane_row + (size_t)row0 * p.d;
+                    const int rows_left = p.N - row0;
+#pragma unroll
+                    for (int k = 0; k < KT; ++k) {
+                        if (k < ntail) {
+#pragma unroll
+                            for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
+                                const bool v = lane + 32 * rp < rows_left;
+                                const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
+                                ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[2], v ? 16u : 0u);
+                                ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[3], v ? 16u : 0u);
+                            }
+                        }
+                    }
+                    ptx::cp_async_commit();
+                    owner_pend = true;
+                }
+            }
             for (int j = 0; j < T; ++j) {
                 if constexpr (HAS_CP) {
                     // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
@@ -569,6 +653,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 }
                 if (++s == S) { s = 0; ph ^= 1; }
             }
+            }
             if (HAS_CP) {
                 ptx::cp_async_wait<0>();  // nothing of ours stays in flight
                 if (ok && pend_s >= 0) {
@@ -579,37 +664,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 }
             }
         };
-        if (warp == 0) {
-            if constexpr (NPAIR == 2) {
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
-                    ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
-                    ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
-                }
-                if constexpr (NA == 2) {
-                    const __nv_bfloat16* o2 = p.own[2] + lane_row + (size_t)row0 * p.d;
-                    const __nv_bfloat16* o3 = p.own[3] + lane_row + (size_t)row0 * p.d;
-                    const int rows_left = p.N - row0;
-#pragma unroll
-                    for (int k = 0; k < KT; ++k) {
-                        if (k < ntail) {
-#pragma unroll
-                            for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
-                                const bool v = lane + 32 * rp < rows_left;
-                                const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
-                                ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[2], v ? 16u : 0u);
-                                ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[3], v ? 16u : 0u);
-                            }
-                        }
-                    }
-                    ptx::cp_async_commit();
-                    owner_pend = true;  // signalled with the first tile's copies: nothing needs them earlier
-                }
-            }
-            produce(std::integral_constant<int, 0>{});
-        } else {
-            produce(std::integral_constant<int, 1>{});
-        }
+        if (warp == 0) produce(std::integral_constant<int, 0>{});
+        else produce(std::integral_constant<int, 1>{});
     } else if (warp == 1 || warp == 3) {
         // ------------------------------------------------------------------ MMA issuers, warps 1 and 3: each
         // whole warp runs its loop in converged control flow; one elected lane issues (see mma_ts_elect).
@@ -637,13 +693,18 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             return kk < 4 ? ptx::smem_desc_sw128(base, 16, 1024) + (uint64_t)((kk * 32) >> 4)
                           : ptx::smem_desc_nosw(base + BWD_ROWS * 128, BWD_ROWS * 16, 128);
         };
-        auto issue_scores = [&](int j, bool) -> bool {
-            const int b = j & 1;
-            if (!ptx::mbar_wait_warp(bar(C::B_EFULL + j % SE), (j / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+        // tiles this CTA streams over all of its items; tile g belongs to item g / T of this CTA
+        const int n_it = (int)blockIdx.x < items ? (items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+        const int G = n_it * T;
+        auto issue_scores = [&](int g) -> bool {  // DV only (the two-pair passes have their own loop below)
+            const int b = g & 1, it = g / T, j = g - it * T;
+            if (!ptx::mbar_wait_warp(bar(C::B_EFULL + g % SE), (g / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            // the first tiles of an item: its owner operands are in tensor memory
+            if (j < 2 && !ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
-            if (lane == 0) BTL_STAMP(0, j, 0);
-            // DV only (the two-pair passes have their own loops below): Y0, Y1 in the E ring, K-major B
-            const uint32_t t0 = tile_addr(0, j), t1 = tile_addr(1, j);
+            if (lane == 0) BTL_STAMP(0, g, 0);
+            // Y0, Y1 in the E ring, K-major B
+            const uint32_t t0 = tile_addr(0, g), t1 = tile_addr(1, g);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk)  // S = X0 Y0^T
@@ -655,23 +716,25 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             for (int kk = 0; kk < KS; ++kk)  // Sd += X0 Y1^T
                 ptx::mma_ts_elect(dT, ax0 + 8 * kk, e_kdesc(t1, kk), idesc_s, 1u);
             ptx::mma_commit_elect(bar(C::B_SFULL + b));
-            ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
-            if (lane == 0) BTL_STAMP(0, j, 1);
+            ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
+            if (lane == 0) BTL_STAMP(0, g, 1);
             return true;
         };
-        auto issue_outputs = [&](int j, bool) -> bool {  // DV only
-            const int b = j & 1;
-            if (lane == 0) BTL_STAMP(0, j, 2);
-            if (!ptx::mbar_wait_warp(bar(C::B_LFULL + j % SL), (j / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-            if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (j >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
-            // the other issuer has queued its batch of tile j - 1: accumulation order is the tile order
-            if (!ptx::turn_wait_warp(turn_addr, (uint32_t)j, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+        auto issue_outputs = [&](int g) -> bool {  // DV only
+            const int b = g & 1, it = g / T, j = g - it * T;
+            if (lane == 0) BTL_STAMP(0, g, 2);
+            if (!ptx::mbar_wait_warp(bar(C::B_LFULL + g % SL), (g / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (g >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            // the other issuer has queued its batch of tile g - 1: accumulation order is the tile order
+            if (!ptx::turn_wait_warp(turn_addr, (uint32_t)g, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            // the first tile of an item overwrites the accumulators: all sixteen element-wise warps have read them
+            if (j == 0 && it > 0 && !ptx::mbar_wait_warp(bar(C::B_ACCFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
-            if (lane == 0) BTL_STAMP(0, j, 3);
+            if (lane == 0) BTL_STAMP(0, g, 3);
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B (the L ring): atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
-            const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);
-            const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
+            const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);
+            const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
 #pragma unroll
             for (int u = 0; u < BC / 16; ++u) {
@@ -681,37 +744,34 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc_o, acc);   // acc1 += A1 B0
                 ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, 1u);    // acc1 += A0 B1
             }
-            ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
+            ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
-            if (lane == 0) BTL_STAMP(0, j, 4);
+            if (lane == 0) BTL_STAMP(0, g, 4);
             return true;
         };
-        bool ok = ptx::mbar_wait_warp(bar(C::B_QREADY), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-        ptx::tc_fence_after_sync();
+        bool ok = true;
         if constexpr (NPAIR == 1) {
-            // warp `wsel` owns the tiles j = wsel, wsel + 2, ...: S(j), then per tile outputs(j) and S(j + 2)
-            if (ok && wsel < T) ok = issue_scores(wsel, false);
-            // The turn passes on after the whole batch (outputs(j), S(j + 2)): two batches queued at once
+            // warp `wsel` owns the tiles g = wsel, wsel + 2, ...: S(g), then per tile outputs(g) and S(g + 2)
+            if (wsel < G) ok = issue_scores(wsel);
+            // The turn passes on after the whole batch (outputs(g), S(g + 2)): two batches queued at once
             // would share the pipe MMA by MMA, both would finish late and together, and the element-wise
             // work of the two buffers would then run back to back instead of under the other's MMAs.
-            for (int j = wsel; ok && j < T; j += 2) {
-                ok = issue_outputs(j, false);  // waits for the L tile, the operands and its turn
-                if (ok && j + 2 < T) ok = issue_scores(j + 2, false);
+            for (int g = wsel; ok && g < G; g += 2) {
+                ok = issue_outputs(g);  // waits for the L tile, the operands and its turn
+                if (ok && g + 2 < G) ok = issue_scores(g + 2);
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)j + 1u);
+                if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)g + 1u);
             }
         } else {
             if (wsel == 0) {  // one issuer: splitting these steps over two warps measured 1 to 2 % slower
-                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-                ptx::tc_fence_after_sync();
                 // One score buffer used in two phases.  Order on the tensor pipe:
                 //   (S, Sd)(0), (D, X)(0), then per tile j: (S, Sd)(j+1) once the element-wise warps have read
                 //   (S, Sd)(j) | outputs(j) once the operands W, dA are written | (D, X)(j+1), which overwrites them.
                 const uint32_t dS = tb + C::COL_SCORE, dT = dS + BC, dD = dS + 2 * BC, dX = dS + 3 * BC;
-                auto issue_first_pair = [&](int j) {  // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; Y0, Y1 in the L ring, K-major
-                    const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, j), 16, 1024);
-                    const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, j), 16, 1024);
+                auto issue_first_pair = [&](int g) {  // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; Y0, Y1 in the L ring, K-major
+                    const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, g), 16, 1024);
+                    const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, g), 16, 1024);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
                         const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
@@ -729,8 +789,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     }
                     ptx::mma_commit_elect(bar(C::B_SFULL + 0));
                 };
-                auto issue_second_pair = [&](int j) {  // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; Y2, Y3 in the E ring
-                    const uint32_t t2 = tile_addr(0, j), t3 = tile_addr(1, j);
+                // `last`: the item's last tile; the shared-memory owner tiles are free once these MMAs are done
+                auto issue_second_pair = [&](int g, bool last) {  // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; Y2, Y3 in the E ring
+                    const uint32_t t2 = tile_addr(0, g), t3 = tile_addr(1, g);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dD, own_kdesc(0, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
@@ -738,60 +799,71 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(0, kk), e_kdesc(t3, kk), idesc_s, 1u);
                     ptx::mma_commit_elect(bar(C::B_SFULL + 1));
-                    ptx::mma_commit_elect(bar(C::B_EEMPTY + j % SE));
+                    ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
+                    if (last) ptx::mma_commit_elect(bar(C::B_OWNFREE));
                 };
-                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + 0), 0, abort_flag, BWD_WAIT_LIMIT_NS);
-                if (ok) {
-                    ptx::tc_fence_after_sync();
-                    issue_first_pair(0);
-                    issue_second_pair(0);
-                }
-                for (int j = 0; ok && j < T; ++j) {
-                    if (j + 1 < T) {
-                        const int jn = j + 1;
-                        // (S, Sd)(j) read by all element-wise warps, and the tiles of j+1 loaded
-                        const bool ready = ptx::mbar_test3_warp(bar(C::B_PREADY + 1), j & 1, bar(C::B_LFULL + jn % SL), (jn / SL) & 1,
-                                                                bar(C::B_EFULL + jn % SE), (jn / SE) & 1);
-                        if (!ready) {
-                            ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + jn % SL), (jn / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + jn % SE), (jn / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                            if (!ok) break;
-                        }
-                        ptx::tc_fence_after_sync();
-                        if (lane == 0) BTL_STAMP(0, jn, 0);
-                        issue_first_pair(jn);
-                        if (lane == 0) BTL_STAMP(0, jn, 1);
-                    }
-                    // outputs(j): acc0 += W B0, acc1 += dA B0 + W B1 with the operands in the D and X columns
-                    if (lane == 0) BTL_STAMP(0, j, 2);
-                    ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), j & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                for (int it = 0; ok && it < n_it; ++it) {
+                    const int g0 = it * T;
+                    // the item's owner operands: X0, X1 in tensor memory, X2, X3 in shared memory
+                    ok = ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    if (ok) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    // (S, Sd) of the tile before, the last of the item before, read by all element-wise warps
+                    if (ok && it > 0) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), (g0 - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + g0 % SL), (g0 / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + g0 % SE), (g0 / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    if (lane == 0) BTL_STAMP(0, j, 3);
-                    {
-                        const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, j), BC * 128, 1024);  // MN-major B
-                        const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, j), BC * 128, 1024);
-                        const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
-#pragma unroll
-                        for (int u = 0; u < BC / 16; ++u) {
-                            const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
-                            const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                            ptx::mma_ts_elect(acc0, dD + 16 * u, b0 + off, idesc_o, acc);
-                            ptx::mma_ts_elect(acc1, dX + 16 * u, b0 + off, idesc_o, acc);
-                            ptx::mma_ts_elect(acc1, dD + 16 * u, b1 + off, idesc_o, 1u);
+                    issue_first_pair(g0);
+                    issue_second_pair(g0, T == 1);
+                    for (int j = 0; ok && j < T; ++j) {
+                        const int g = g0 + j;
+                        if (j + 1 < T) {
+                            const int gn = g + 1;
+                            // (S, Sd)(g) read by all element-wise warps, and the tiles of g+1 loaded
+                            const bool ready = ptx::mbar_test3_warp(bar(C::B_PREADY + 1), g & 1, bar(C::B_LFULL + gn % SL), (gn / SL) & 1,
+                                                                    bar(C::B_EFULL + gn % SE), (gn / SE) & 1);
+                            if (!ready) {
+                                ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_LFULL + gn % SL), (gn / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + gn % SE), (gn / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                                if (!ok) break;
+                            }
+                            ptx::tc_fence_after_sync();
+                            if (lane == 0) BTL_STAMP(0, gn, 0);
+                            issue_first_pair(gn);
+                            if (lane == 0) BTL_STAMP(0, gn, 1);
                         }
-                        ptx::mma_commit_elect(bar(C::B_LEMPTY + j % SL));
-                        if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                        // outputs(g): acc0 += W B0, acc1 += dA B0 + W B1 with the operands in the D and X columns
+                        if (lane == 0) BTL_STAMP(0, g, 2);
+                        ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), g & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        // the first tile of an item overwrites the accumulators: the element-wise warps have read them
+                        if (ok && j == 0 && it > 0) ok = ptx::mbar_wait_warp(bar(C::B_ACCFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
+                        if (lane == 0) BTL_STAMP(0, g, 3);
+                        {
+                            const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);  // MN-major B
+                            const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
+                            const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+#pragma unroll
+                            for (int u = 0; u < BC / 16; ++u) {
+                                const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                                const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                                ptx::mma_ts_elect(acc0, dD + 16 * u, b0 + off, idesc_o, acc);
+                                ptx::mma_ts_elect(acc1, dX + 16 * u, b0 + off, idesc_o, acc);
+                                ptx::mma_ts_elect(acc1, dD + 16 * u, b1 + off, idesc_o, 1u);
+                            }
+                            ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
+                            if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                        }
+                        if (lane == 0) BTL_STAMP(0, g, 4);
+                        if (j + 1 < T) issue_second_pair(g + 1, j + 2 == T);
                     }
-                    if (lane == 0) BTL_STAMP(0, j, 4);
-                    if (j + 1 < T) issue_second_pair(j + 1);
                 }
             }
         }
     } else {
-        bwd_elementwise<MODE, DP>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, bh, row0, T);
+        bwd_elementwise<MODE, DP>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, items, row_tiles, T);
     }
 
     // ---------------------------------------------------------------------- teardown

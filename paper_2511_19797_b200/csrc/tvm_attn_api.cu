@@ -245,7 +245,13 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
     auto kern = jvp_bwd_kernel<MODE, DP>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
         return TVM_ATTN_CUDA_ERROR;
-    const long long grid = s.BH * ((s.N + BWD_ROWS - 1) / BWD_ROWS);
+    // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
+    // items go round-robin over them
+    const long long items = s.BH * ((s.N + BWD_ROWS - 1) / BWD_ROWS);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return TVM_ATTN_CUDA_ERROR;
+    const long long grid = items < sms ? items : sms;
     g_prof.before(st);
     {
         // DK and DQ read nothing that the pass before them writes (DV, DK and DQ all depend on the row-sums
