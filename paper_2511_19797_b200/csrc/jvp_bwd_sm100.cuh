@@ -217,186 +217,186 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     int it = 0;  // items done by this CTA
     if ((int)blockIdx.x < items) stage_x(blockIdx.x);
     for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
-    const int g0 = it * T;  // tiles this CTA has streamed before this item: rings and barrier phases run on
-    const int bh = item / row_tiles;
-    const int row0 = (item - bh * row_tiles) * BWD_ROWS;
-    const bool row_valid = row0 + row < p.N;
-    const size_t grow = (size_t)bh * p.N + row0 + row;
-    float r_lse2 = CUDART_INF_F, r_mu = 0.f, r_s1 = 0.f, r_cv = 0.f;  // per-row statistics (DQ)
-    if (MODE == BWD_DQ && row_valid) {
-        r_lse2 = p.lse2[grow];
-        r_mu = p.mu[grow];
-        r_s1 = p.sig1[grow];
-        r_cv = p.cvec[grow];
-    }
-    for (int j = NPAIR == 1 ? ((par ^ g0) & 1) : 0; j < T; j += jstep) {
-        const int g = g0 + j;
-        const int b = NPAIR == 1 ? (g & 1) : 0, sph = NPAIR == 1 ? (g >> 1) & 1 : (g & 1);
-        if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        // the statistics of the tile's queries arrive with its L stage, which is not released before the
-        // output MMAs of this tile, hence not before every warp is through with them
-        const float* st = stats + (g % C::SL) * 4 * 64 + 16 * sl;
-        if (C::TRANSPOSED)
-            if (!ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        ptx::tc_fence_after_sync();
-        if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 0);
-        const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
-        const int key0 = j * BC + 16 * sl;  // first stream row of this slice
-        if (NPAIR == 1) {
-          const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
+        const int g0 = it * T;  // tiles this CTA has streamed before this item: rings and barrier phases run on
+        const int bh = item / row_tiles;
+        const int row0 = (item - bh * row_tiles) * BWD_ROWS;
+        const bool row_valid = row0 + row < p.N;
+        const size_t grow = (size_t)bh * p.N + row0 + row;
+        float r_lse2 = CUDART_INF_F, r_mu = 0.f, r_s1 = 0.f, r_cv = 0.f;  // per-row statistics (DQ)
+        if (MODE == BWD_DQ && row_valid) {
+            r_lse2 = p.lse2[grow];
+            r_mu = p.mu[grow];
+            r_s1 = p.sig1[grow];
+            r_cv = p.cvec[grow];
+        }
+        for (int j = NPAIR == 1 ? ((par ^ g0) & 1) : 0; j < T; j += jstep) {
+            const int g = g0 + j;
+            const int b = NPAIR == 1 ? (g & 1) : 0, sph = NPAIR == 1 ? (g >> 1) & 1 : (g & 1);
+            if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            // the statistics of the tile's queries arrive with its L stage, which is not released before the
+            // output MMAs of this tile, hence not before every warp is through with them
+            const float* st = stats + (g % C::SL) * 4 * 64 + 16 * sl;
+            if (C::TRANSPOSED)
+                if (!ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 0);
+            const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
+            const int key0 = j * BC + 16 * sl;  // first stream row of this slice
+            if (NPAIR == 1) {
+              const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
 #pragma unroll
-          for (int sub = 0; sub < 2; ++sub) {  // this warp's two slices
-            const uint32_t sb = sbase + 16 * sub;
-            const float* stt = st + 16 * sub;
-            uint32_t s1[16], s2[16];
-            ptx::tmem_ld16(sb, s1);
-            ptx::tmem_ld16(sb + BC, s2);
-            ptx::tmem_wait_ld();
-            uint32_t pa0[8], pa1[8];
-#pragma unroll
-            for (int c4 = 0; c4 < 16; c4 += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(stt + c4);
-                const float4 m4 = *reinterpret_cast<const float4*>(stt + 64 + c4);
-                const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
-#pragma unroll
-                for (int e = 0; e < 4; e += 2) {  // P = 2^(c2 s - lse2), P Nn with Nn = alpha ts - mu: two columns per instruction
-                    const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
-                    float x0, x1;
-                    ptx::unpack2(x2, x0, x1);
-                    const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
-                    const uint64_t n2 = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
-                    const uint64_t q2 = ptx::mul2(ptx::pack2(p0, p1), n2);
-                    float q0, q1;
-                    ptx::unpack2(q2, q0, q1);
-                    pa0[(c4 + e) >> 1] = ptx::pack_bf16(p0, p1);
-                    pa1[(c4 + e) >> 1] = ptx::pack_bf16(q0, q1);
-                }
-            }
-            // operand of a k-step (16 stream rows) sits at the slice's columns of the accumulator it replaces
-            ptx::tmem_st8(sb, pa0);
-            ptx::tmem_st8(sb + BC, pa1);
-          }
-        } else {
-            // ---- phase A: P, Nn, -P Sigma1, -P c from (S, Sd), two columns per register pair; then that half of the
-            // buffer may be overwritten.  Phase B, which sits on the critical path between the second score pair and
-            // the output MMAs, is left with three packed FMAs per column pair.
-            uint64_t P2[8], Nn2[8], nPs2[8], nPc2[8];
-            {
+              for (int sub = 0; sub < 2; ++sub) {  // this warp's two slices
+                const uint32_t sb = sbase + 16 * sub;
+                const float* stt = st + 16 * sub;
                 uint32_t s1[16], s2[16];
-                ptx::tmem_ld16(sbase, s1);
-                ptx::tmem_ld16(sbase + BC, s2);
+                ptx::tmem_ld16(sb, s1);
+                ptx::tmem_ld16(sb + BC, s2);
                 ptx::tmem_wait_ld();
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + 1));
-                const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
+                uint32_t pa0[8], pa1[8];
 #pragma unroll
                 for (int c4 = 0; c4 < 16; c4 += 4) {
-                    float lv[4], mv[4], gv[4], cv[4];
-                    if (C::TRANSPOSED) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
-                        const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
-                        const float4 g4 = *reinterpret_cast<const float4*>(st + 128 + c4);
-                        const float4 c44 = *reinterpret_cast<const float4*>(st + 192 + c4);
-                        lv[0] = l4.x; lv[1] = l4.y; lv[2] = l4.z; lv[3] = l4.w;
-                        mv[0] = m4.x; mv[1] = m4.y; mv[2] = m4.z; mv[3] = m4.w;
-                        gv[0] = g4.x; gv[1] = g4.y; gv[2] = g4.z; gv[3] = g4.w;
-                        cv[0] = c44.x; cv[1] = c44.y; cv[2] = c44.z; cv[3] = c44.w;
-                    } else {
+                    const float4 l4 = *reinterpret_cast<const float4*>(stt + c4);
+                    const float4 m4 = *reinterpret_cast<const float4*>(stt + 64 + c4);
+                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            lv[e] = (key0 + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
-                            mv[e] = r_mu; gv[e] = r_s1; cv[e] = r_cv;
-                        }
-                    }
-#pragma unroll
-                    for (int e = 0; e < 4; e += 2) {
-                        const int k = (c4 + e) >> 1;
+                    for (int e = 0; e < 4; e += 2) {  // P = 2^(c2 s - lse2), P Nn with Nn = alpha ts - mu: two columns per instruction
                         const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
                         float x0, x1;
                         ptx::unpack2(x2, x0, x1);
-                        P2[k] = ptx::pack2(ptx::ex2(x0), ptx::ex2(x1));
-                        Nn2[k] = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
-                        nPs2[k] = ptx::mul2(P2[k], ptx::pack2(-gv[e], -gv[e + 1]));
-                        nPc2[k] = ptx::mul2(P2[k], ptx::pack2(-cv[e], -cv[e + 1]));
+                        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                        const uint64_t n2 = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
+                        const uint64_t q2 = ptx::mul2(ptx::pack2(p0, p1), n2);
+                        float q0, q1;
+                        ptx::unpack2(q2, q0, q1);
+                        pa0[(c4 + e) >> 1] = ptx::pack_bf16(p0, p1);
+                        pa1[(c4 + e) >> 1] = ptx::pack_bf16(q0, q1);
+                    }
+                }
+                // operand of a k-step (16 stream rows) sits at the slice's columns of the accumulator it replaces
+                ptx::tmem_st8(sb, pa0);
+                ptx::tmem_st8(sb + BC, pa1);
+              }
+            } else {
+                // ---- phase A: P, Nn, -P Sigma1, -P c from (S, Sd), two columns per register pair; then that half of the
+                // buffer may be overwritten.  Phase B, which sits on the critical path between the second score pair and
+                // the output MMAs, is left with three packed FMAs per column pair.
+                uint64_t P2[8], Nn2[8], nPs2[8], nPc2[8];
+                {
+                    uint32_t s1[16], s2[16];
+                    ptx::tmem_ld16(sbase, s1);
+                    ptx::tmem_ld16(sbase + BC, s2);
+                    ptx::tmem_wait_ld();
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + 1));
+                    const uint64_t c2c2 = ptx::pack2(p.c2, p.c2), aa = ptx::pack2(p.alpha, p.alpha);
+#pragma unroll
+                    for (int c4 = 0; c4 < 16; c4 += 4) {
+                        float lv[4], mv[4], gv[4], cv[4];
+                        if (C::TRANSPOSED) {
+                            const float4 l4 = *reinterpret_cast<const float4*>(st + c4);
+                            const float4 m4 = *reinterpret_cast<const float4*>(st + 64 + c4);
+                            const float4 g4 = *reinterpret_cast<const float4*>(st + 128 + c4);
+                            const float4 c44 = *reinterpret_cast<const float4*>(st + 192 + c4);
+                            lv[0] = l4.x; lv[1] = l4.y; lv[2] = l4.z; lv[3] = l4.w;
+                            mv[0] = m4.x; mv[1] = m4.y; mv[2] = m4.z; mv[3] = m4.w;
+                            gv[0] = g4.x; gv[1] = g4.y; gv[2] = g4.z; gv[3] = g4.w;
+                            cv[0] = c44.x; cv[1] = c44.y; cv[2] = c44.z; cv[3] = c44.w;
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                lv[e] = (key0 + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
+                                mv[e] = r_mu; gv[e] = r_s1; cv[e] = r_cv;
+                            }
+                        }
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            const int k = (c4 + e) >> 1;
+                            const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
+                            float x0, x1;
+                            ptx::unpack2(x2, x0, x1);
+                            P2[k] = ptx::pack2(ptx::ex2(x0), ptx::ex2(x1));
+                            Nn2[k] = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
+                            nPs2[k] = ptx::mul2(P2[k], ptx::pack2(-gv[e], -gv[e + 1]));
+                            nPc2[k] = ptx::mul2(P2[k], ptx::pack2(-cv[e], -cv[e + 1]));
+                        }
+                    }
+                }
+                // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 2);
+                if (!ptx::mbar_wait(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 3);
+                uint32_t s3[16], s4[16];
+                ptx::tmem_ld16(sbase + 2 * BC, s3);
+                ptx::tmem_ld16(sbase + 3 * BC, s4);
+                ptx::tmem_wait_ld();
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 4);
+                uint32_t pa0[8], pa1[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint64_t w2 = ptx::fma2(P2[k], ptx::pack2u(s3[2 * k], s3[2 * k + 1]), nPs2[k]);
+                    const uint64_t t2 = ptx::fma2(P2[k], ptx::pack2u(s4[2 * k], s4[2 * k + 1]), nPc2[k]);
+                    const uint64_t d2 = ptx::fma2(w2, Nn2[k], t2);
+                    float w0, w1, d0, d1;
+                    ptx::unpack2(w2, w0, w1);
+                    ptx::unpack2(d2, d0, d1);
+                    pa0[k] = ptx::pack_bf16(w0, w1);
+                    pa1[k] = ptx::pack_bf16(d0, d1);
+                }
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 5);
+                ptx::tmem_st8(sbase + 2 * BC, pa0);
+                ptx::tmem_st8(sbase + 3 * BC, pa1);
+            }
+            ptx::tmem_wait_st();
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 6);
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);
+            if (lane == 0) BTL_STAMP(4 + (w >> 3), j, w & 7);
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
+        }
+        if (!ok) break;
+        // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
+        if (item + (int)gridDim.x < items) {
+            if (NPAIR == 1) {
+                // DV: this warp has seen only the scores of its own tiles; those of the item's last tile, which
+                // may belong to the other eight warps, must be complete too before the operands change
+                const int gl = g0 + T - 1;
+                if (!ptx::mbar_wait(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            }
+            stage_x(item + gridDim.x);
+        }
+        if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            __nv_bfloat16* p0 = p.out0 + grow * p.d;
+            __nv_bfloat16* p1 = p.out1 + grow * p.d;
+            for (int ch = slot; ch < KS; ch += 4) {
+                uint32_t x0[16], x1[16];
+                ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, x0);
+                ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, x1);
+                ptx::tmem_wait_ld();
+                uint32_t q0[8], q1[8];
+#pragma unroll
+                for (int c = 0; c < 16; c += 2) {
+                    q0[c >> 1] = ptx::pack_bf16(__uint_as_float(x0[c]) * p.out_scale, __uint_as_float(x0[c + 1]) * p.out_scale);
+                    q1[c >> 1] = ptx::pack_bf16(__uint_as_float(x1[c]) * p.out_scale, __uint_as_float(x1[c + 1]) * p.out_scale);
+                }
+                if (row_valid) {
+                    *reinterpret_cast<uint4*>(p0 + 16 * ch) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
+                    *reinterpret_cast<uint4*>(p1 + 16 * ch) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
+                    if (16 * ch + 8 < p.d) {
+                        *reinterpret_cast<uint4*>(p0 + 16 * ch + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
+                        *reinterpret_cast<uint4*>(p1 + 16 * ch + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
                     }
                 }
             }
-            // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 2);
-            if (!ptx::mbar_wait(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
-            ptx::tc_fence_after_sync();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 3);
-            uint32_t s3[16], s4[16];
-            ptx::tmem_ld16(sbase + 2 * BC, s3);
-            ptx::tmem_ld16(sbase + 3 * BC, s4);
-            ptx::tmem_wait_ld();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 4);
-            uint32_t pa0[8], pa1[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint64_t w2 = ptx::fma2(P2[k], ptx::pack2u(s3[2 * k], s3[2 * k + 1]), nPs2[k]);
-                const uint64_t t2 = ptx::fma2(P2[k], ptx::pack2u(s4[2 * k], s4[2 * k + 1]), nPc2[k]);
-                const uint64_t d2 = ptx::fma2(w2, Nn2[k], t2);
-                float w0, w1, d0, d1;
-                ptx::unpack2(w2, w0, w1);
-                ptx::unpack2(d2, d0, d1);
-                pa0[k] = ptx::pack_bf16(w0, w1);
-                pa1[k] = ptx::pack_bf16(d0, d1);
-            }
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 5);
-            ptx::tmem_st8(sbase + 2 * BC, pa0);
-            ptx::tmem_st8(sbase + 3 * BC, pa1);
+            // the accumulators may be overwritten by the first output MMAs of the next item
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_ACCFREE));
         }
-        ptx::tmem_wait_st();
-        if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 6);
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);
-        if (lane == 0) BTL_STAMP(4 + (w >> 3), j, w & 7);
-        if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
-    }
-    if (!ok) break;
-    // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
-    if (item + (int)gridDim.x < items) {
-        if (NPAIR == 1) {
-            // DV: this warp has seen only the scores of its own tiles; those of the item's last tile, which
-            // may belong to the other eight warps, must be complete too before the operands change
-            const int gl = g0 + T - 1;
-            if (!ptx::mbar_wait(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        }
-        stage_x(item + gridDim.x);
-    }
-    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-    if (ok) {
-        ptx::tc_fence_after_sync();
-        __nv_bfloat16* p0 = p.out0 + grow * p.d;
-        __nv_bfloat16* p1 = p.out1 + grow * p.d;
-        for (int ch = slot; ch < KS; ch += 4) {
-            uint32_t x0[16], x1[16];
-            ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, x0);
-            ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, x1);
-            ptx::tmem_wait_ld();
-            uint32_t q0[8], q1[8];
-#pragma unroll
-            for (int c = 0; c < 16; c += 2) {
-                q0[c >> 1] = ptx::pack_bf16(__uint_as_float(x0[c]) * p.out_scale, __uint_as_float(x0[c + 1]) * p.out_scale);
-                q1[c >> 1] = ptx::pack_bf16(__uint_as_float(x1[c]) * p.out_scale, __uint_as_float(x1[c + 1]) * p.out_scale);
-            }
-            if (row_valid) {
-                *reinterpret_cast<uint4*>(p0 + 16 * ch) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
-                *reinterpret_cast<uint4*>(p1 + 16 * ch) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
-                if (16 * ch + 8 < p.d) {
-                    *reinterpret_cast<uint4*>(p0 + 16 * ch + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
-                    *reinterpret_cast<uint4*>(p1 + 16 * ch + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
-                }
-            }
-        }
-        // the accumulators may be overwritten by the first output MMAs of the next item
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar(C::B_ACCFREE));
-    }
     }
 }
 
@@ -524,135 +524,135 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
             int it = 0;
             for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
-            const int bh = item / row_tiles;
-            [[maybe_unused]] const int row0 = (item - bh * row_tiles) * BWD_ROWS;
-            [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
-            [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
-            [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
-            [[maybe_unused]] const size_t srow = (size_t)bh * p.N;
-            [[maybe_unused]] const float* st_src0 = (lane < 16 ? p.lse2 : p.mu) + srow + 4 * (lane & 15);
-            [[maybe_unused]] const float* st_src1 = NST == 4 ? (lane < 16 ? p.sig1 : p.cvec) + srow + 4 * (lane & 15) : nullptr;
-            if constexpr (ring == 0 && NPAIR == 2) {
-                // The shared-memory owner tiles of this item, once the MMAs that read those of the item before
-                // are done.  Their copied columns are signalled with the first tile's: nothing needs them earlier.
-                if (it > 0) {
+                const int bh = item / row_tiles;
+                [[maybe_unused]] const int row0 = (item - bh * row_tiles) * BWD_ROWS;
+                [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
+                [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
+                [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
+                [[maybe_unused]] const size_t srow = (size_t)bh * p.N;
+                [[maybe_unused]] const float* st_src0 = (lane < 16 ? p.lse2 : p.mu) + srow + 4 * (lane & 15);
+                [[maybe_unused]] const float* st_src1 = NST == 4 ? (lane < 16 ? p.sig1 : p.cvec) + srow + 4 * (lane & 15) : nullptr;
+                if constexpr (ring == 0 && NPAIR == 2) {
+                    // The shared-memory owner tiles of this item, once the MMAs that read those of the item before
+                    // are done.  Their copied columns are signalled with the first tile's: nothing needs them earlier.
+                    if (it > 0) {
+                        if constexpr (HAS_CP) {
+                            // the MMAs waited for below need the last tile of the item before: signal its copies first
+                            if (pend_s >= 0) {
+                                ptx::cp_async_wait<0>();
+                                ptx::fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                                pend_s = -1;
+                            }
+                        }
+                        ok = ptx::mbar_wait_warp(bar(C::B_OWNFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        if (!ok) break;
+                    }
+                    if (lane == 0) {
+                        ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
+                        ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
+                        ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
+                    }
+                    if constexpr (NA == 2) {
+                        const __nv_bfloat16* o2 = p.own[2] + lane_row + (size_t)row0 * p.d;
+                        const __nv_bfloat16* o3 = p.own[3] + lane_row + (size_t)row0 * p.d;
+                        const int rows_left = p.N - row0;
+#pragma unroll
+                        for (int k = 0; k < KT; ++k) {
+                            if (k < ntail) {
+#pragma unroll
+                                for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
+                                    const bool v = lane + 32 * rp < rows_left;
+                                    const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
+                                    ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[2], v ? 16u : 0u);
+                                    ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[3], v ? 16u : 0u);
+                                }
+                            }
+                        }
+                        ptx::cp_async_commit();
+                        owner_pend = true;
+                    }
+                }
+                for (int j = 0; j < T; ++j) {
                     if constexpr (HAS_CP) {
-                        // the MMAs waited for below need the last tile of the item before: signal its copies first
-                        if (pend_s >= 0) {
+                        // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
+                        // that tile before it frees the stage.
+                        if (pend_s >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
                             ptx::cp_async_wait<0>();
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                            if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 3);
                             pend_s = -1;
+                            if (ring == 0 && owner_pend) {  // cp.async groups complete in order: the owner copies have landed too
+                                if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+                                owner_pend = false;
+                            }
                         }
                     }
-                    ok = ptx::mbar_wait_warp(bar(C::B_OWNFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     if (!ok) break;
-                }
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
-                    ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
-                    ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
-                }
-                if constexpr (NA == 2) {
-                    const __nv_bfloat16* o2 = p.own[2] + lane_row + (size_t)row0 * p.d;
-                    const __nv_bfloat16* o3 = p.own[3] + lane_row + (size_t)row0 * p.d;
-                    const int rows_left = p.N - row0;
-#pragma unroll
-                    for (int k = 0; k < KT; ++k) {
-                        if (k < ntail) {
-#pragma unroll
-                            for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
-                                const bool v = lane + 32 * rp < rows_left;
-                                const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
-                                ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[2], v ? 16u : 0u);
-                                ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[3], v ? 16u : 0u);
+                    if (lane == 0 && ring == 0) BTL_STAMP(2, j, 0);
+                    const uint32_t stage = ring_base + s * 2 * TB;
+                    if (lane == 0) {
+                        ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
+                        ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
+                        ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
+                    }
+                    if constexpr (HAS_CP) {
+                        [[maybe_unused]] const int rows_left = p.N - j * BC;  // rows of this tile that exist
+                        if constexpr (STATS) {
+                            // queries beyond N read as zero: their rows of the B operands are zero too
+                            const uint32_t slot = st_base + s * (4 * 64 * 4);
+                            if (st16) {
+                                const bool v = 4 * (lane & 15) < rows_left;
+                                const uint32_t dst = slot + (lane >> 4) * 256 + (lane & 15) * 16;
+                                ptx::cp_async_16(dst, v ? st_src0 + j * BC : p.lse2, v ? 16u : 0u);
+                                if (NST == 4) ptx::cp_async_16(dst + 512, v ? st_src1 + j * BC : p.lse2, v ? 16u : 0u);
+                            } else {
+                                for (int c = lane; c < NST * 64; c += 32) {
+                                    const int stat = c >> 6, r = c & 63;
+                                    const float* src = (stat == 0 ? p.lse2 : stat == 1 ? p.mu : stat == 2 ? p.sig1 : p.cvec) + srow + j * BC + r;
+                                    const bool v = r < rows_left;
+                                    ptx::cp_async_4(slot + c * 4, v ? src : p.lse2, v ? 4u : 0u);
+                                }
                             }
                         }
-                    }
-                    ptx::cp_async_commit();
-                    owner_pend = true;
-                }
-            }
-            for (int j = 0; j < T; ++j) {
-                if constexpr (HAS_CP) {
-                    // Never block on a free stage while a tile's copies are unsignalled: the consumer may need
-                    // that tile before it frees the stage.
-                    if (pend_s >= 0 && !ptx::mbar_test_warp(bar(b_empty + s), ph ^ 1)) {
-                        ptx::cp_async_wait<0>();
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
-                        if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 3);
-                        pend_s = -1;
-                        if (ring == 0 && owner_pend) {  // cp.async groups complete in order: the owner copies have landed too
-                            if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
-                            owner_pend = false;
-                        }
-                    }
-                }
-                ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
-                if (!ok) break;
-                if (lane == 0 && ring == 0) BTL_STAMP(2, j, 0);
-                const uint32_t stage = ring_base + s * 2 * TB;
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
-                    ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
-                    ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
-                }
-                if constexpr (HAS_CP) {
-                    [[maybe_unused]] const int rows_left = p.N - j * BC;  // rows of this tile that exist
-                    if constexpr (STATS) {
-                        // queries beyond N read as zero: their rows of the B operands are zero too
-                        const uint32_t slot = st_base + s * (4 * 64 * 4);
-                        if (st16) {
-                            const bool v = 4 * (lane & 15) < rows_left;
-                            const uint32_t dst = slot + (lane >> 4) * 256 + (lane & 15) * 16;
-                            ptx::cp_async_16(dst, v ? st_src0 + j * BC : p.lse2, v ? 16u : 0u);
-                            if (NST == 4) ptx::cp_async_16(dst + 512, v ? st_src1 + j * BC : p.lse2, v ? 16u : 0u);
-                        } else {
-                            for (int c = lane; c < NST * 64; c += 32) {
-                                const int stat = c >> 6, r = c & 63;
-                                const float* src = (stat == 0 ? p.lse2 : stat == 1 ? p.mu : stat == 2 ? p.sig1 : p.cvec) + srow + j * BC + r;
-                                const bool v = r < rows_left;
-                                ptx::cp_async_4(slot + c * 4, v ? src : p.lse2, v ? 4u : 0u);
+#pragma unroll
+                        for (int k = 0; k < (NA == 2 ? KT : 0); ++k) {
+                            if (k < ntail) {
+#pragma unroll
+                                for (int rp = 0; rp < BC / 32; ++rp) {
+                                    const bool v = lane + 32 * rp < rows_left;
+                                    const uint32_t dst = stage + dst_lane +
+                                                         (ring == 0 ? k * BC * 16 + rp * 32 * 16 : rp * 32 * 128 + ((k ^ sw) << 4));
+                                    ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
+                                    ptx::cp_async_16(dst + TB, v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                                }
                             }
                         }
-                    }
-#pragma unroll
-                    for (int k = 0; k < (NA == 2 ? KT : 0); ++k) {
-                        if (k < ntail) {
-#pragma unroll
-                            for (int rp = 0; rp < BC / 32; ++rp) {
-                                const bool v = lane + 32 * rp < rows_left;
-                                const uint32_t dst = stage + dst_lane +
-                                                     (ring == 0 ? k * BC * 16 + rp * 32 * 16 : rp * 32 * 128 + ((k ^ sw) << 4));
-                                ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
-                                ptx::cp_async_16(dst + TB, v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                        ptx::cp_async_commit();
+                        if (lane == 0 && ring == 0) BTL_STAMP(2, j, 1);
+                        if (pend_s >= 0) {  // the tile before: its copies have had a whole iteration to land
+                            ptx::cp_async_wait<1>();
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+                            if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 2);
+                            if (ring == 0 && owner_pend) {
+                                if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+                                owner_pend = false;
                             }
                         }
-                    }
-                    ptx::cp_async_commit();
-                    if (lane == 0 && ring == 0) BTL_STAMP(2, j, 1);
-                    if (pend_s >= 0) {  // the tile before: its copies have had a whole iteration to land
-                        ptx::cp_async_wait<1>();
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
-                        if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 2);
-                        if (ring == 0 && owner_pend) {
-                            if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
-                            owner_pend = false;
+                        pend_s = s;
+                        if constexpr (NA == 2) {
+                            src0 += tile_elems;
+                            src1 += tile_elems;
                         }
                     }
-                    pend_s = s;
-                    if constexpr (NA == 2) {
-                        src0 += tile_elems;
-                        src1 += tile_elems;
-                    }
+                    if (++s == S) { s = 0; ph ^= 1; }
                 }
-                if (++s == S) { s = 0; ph ^= 1; }
-            }
             }
             if (HAS_CP) {
                 ptx::cp_async_wait<0>();  // nothing of ours stays in flight

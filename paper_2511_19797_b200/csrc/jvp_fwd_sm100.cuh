@@ -157,190 +157,190 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
     if ((int)blockIdx.x < items) stage_q(blockIdx.x);
 
     for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
-    const int bh = item / row_tiles;
-    const int row0 = (item - bh * row_tiles) * FWD_ROWS;
-    const bool row_valid = row0 + row < p.N;
-    const size_t grow = (size_t)bh * p.N + row0 + row;
-    float m_ref = -CUDART_INF_F, cen = 0.f;
-    uint64_t l2 = 0ull, mt2 = 0ull;  // two partial sums each of P~ and of P~(T - c) over this warp's slices
+        const int bh = item / row_tiles;
+        const int row0 = (item - bh * row_tiles) * FWD_ROWS;
+        const bool row_valid = row0 + row < p.N;
+        const size_t grow = (size_t)bh * p.N + row0 + row;
+        float m_ref = -CUDART_INF_F, cen = 0.f;
+        uint64_t l2 = 0ull, mt2 = 0ull;  // two partial sums each of P~ and of P~(T - c) over this warp's slices
 
-    for (int j = 0; j < T; ++j, ++g) {
-        const int b = g & 1;
-        // S is complete before Sd: the row maxima are found and exchanged while the Sd MMAs still run
-        if (!ptx::mbar_wait(bar(C::B_SFULL + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        ptx::tc_fence_after_sync();
-        const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS;
-        uint32_t s[16], ts[16];
-        ptx::tmem_ld16(sbase + 16 * sl, s);
-        ptx::tmem_wait_ld();
-        const int nvalid = p.N - j * BC - 16 * sl;  // columns of this slice that are real keys
-        if (nvalid < 16) {
+        for (int j = 0; j < T; ++j, ++g) {
+            const int b = g & 1;
+            // S is complete before Sd: the row maxima are found and exchanged while the Sd MMAs still run
+            if (!ptx::mbar_wait(bar(C::B_SFULL + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS;
+            uint32_t s[16], ts[16];
+            ptx::tmem_ld16(sbase + 16 * sl, s);
+            ptx::tmem_wait_ld();
+            const int nvalid = p.N - j * BC - 16 * sl;  // columns of this slice that are real keys
+            if (nvalid < 16) {
 #pragma unroll
-            for (int c = 0; c < 16; ++c)
-                if (c >= nvalid) s[c] = __float_as_uint(-CUDART_INF_F);
-        }
-        // slice maximum, exchanged with the three other warps of this quadrant
-        float mx = ptx::max3(__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(s[2]));
-#pragma unroll
-        for (int c = 3; c < 15; c += 2) mx = ptx::max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-        mx = fmaxf(mx, __uint_as_float(s[15]));
-        float* xm = xmax + (g & 1) * 512;
-        xm[row * 4 + sl] = mx;
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar(C::B_XMAX + q));
-        if (!ptx::mbar_wait(bar(C::B_SFULL + 2 + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        ptx::tc_fence_after_sync();
-        ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
-        if (!ptx::mbar_wait(bar(C::B_XMAX + q), g & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
-        const float4 o4 = *reinterpret_cast<const float4*>(xm + row * 4);
-        const float mrow = fmaxf(ptx::max3(o4.x, o4.y, o4.z), o4.w) * p.c2;  // tile maximum of the row, log2 units
-        ptx::tmem_wait_ld();
-        const bool need = mrow > m_ref + FWD_LAZY_LOG2;
-        if (__any_sync(0xffffffffu, need)) {
-            // ---- slow path, taken by the four warps of the quadrant together
-            float la = -CUDART_INF_F, lt = 0.f;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const bool gt = __uint_as_float(s[c]) > la;
-                la = gt ? __uint_as_float(s[c]) : la;
-                lt = gt ? __uint_as_float(ts[c]) : lt;
+                for (int c = 0; c < 16; ++c)
+                    if (c >= nvalid) s[c] = __float_as_uint(-CUDART_INF_F);
             }
-            xs2[row * 4 + sl] = make_float2(la, lt);
+            // slice maximum, exchanged with the three other warps of this quadrant
+            float mx = ptx::max3(__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(s[2]));
+#pragma unroll
+            for (int c = 3; c < 15; c += 2) mx = ptx::max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+            mx = fmaxf(mx, __uint_as_float(s[15]));
+            float* xm = xmax + (g & 1) * 512;
+            xm[row * 4 + sl] = mx;
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
-            if (!ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
-            ++n_slow;
-            float ba = -CUDART_INF_F, bt = 0.f;
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_XMAX + q));
+            if (!ptx::mbar_wait(bar(C::B_SFULL + 2 + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            ptx::tmem_ld16(sbase + BC + 16 * sl, ts);
+            if (!ptx::mbar_wait(bar(C::B_XMAX + q), g & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            const float4 o4 = *reinterpret_cast<const float4*>(xm + row * 4);
+            const float mrow = fmaxf(ptx::max3(o4.x, o4.y, o4.z), o4.w) * p.c2;  // tile maximum of the row, log2 units
+            ptx::tmem_wait_ld();
+            const bool need = mrow > m_ref + FWD_LAZY_LOG2;
+            if (__any_sync(0xffffffffu, need)) {
+                // ---- slow path, taken by the four warps of the quadrant together
+                float la = -CUDART_INF_F, lt = 0.f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {  // ties go to the lowest slice
-                const float2 v = xs2[row * 4 + k];
-                const bool gt = v.x > ba;
-                ba = gt ? v.x : ba;
-                bt = gt ? v.y : bt;
-            }
-            const float tw = bt * p.alpha;
-            const float scale = need ? ptx::ex2(m_ref - mrow) : 1.0f;
-            const float fix = need ? cen - tw : 0.f;
-            if (need) { m_ref = mrow; cen = tw; }
-            {
-                float l0, l1, t0, t1;
-                ptx::unpack2(l2, l0, l1);
-                ptx::unpack2(mt2, t0, t1);
-                t0 = scale * fmaf(fix, l0, t0);
-                t1 = scale * fmaf(fix, l1, t1);
-                l0 *= scale;
-                l1 *= scale;
-                l2 = ptx::pack2(l0, l1);
-                mt2 = ptx::pack2(t0, t1);
-            }
-            if (j > 0) {
-                // accumulators must be at rest: the value MMAs of tile j-1 have completed
-                if (!ptx::mbar_wait(bar(C::B_OUTDONE + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
-                ptx::tc_fence_after_sync();
-                // eight columns at a time: this rare path must not set the register peak of the loop
-                for (int ch = 2 * sl; ch < 2 * KS; ch += 8) {
+                for (int c = 0; c < 16; ++c) {
+                    const bool gt = __uint_as_float(s[c]) > la;
+                    la = gt ? __uint_as_float(s[c]) : la;
+                    lt = gt ? __uint_as_float(ts[c]) : lt;
+                }
+                xs2[row * 4 + sl] = make_float2(la, lt);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
+                if (!ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                ++n_slow;
+                float ba = -CUDART_INF_F, bt = 0.f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {  // ties go to the lowest slice
+                    const float2 v = xs2[row * 4 + k];
+                    const bool gt = v.x > ba;
+                    ba = gt ? v.x : ba;
+                    bt = gt ? v.y : bt;
+                }
+                const float tw = bt * p.alpha;
+                const float scale = need ? ptx::ex2(m_ref - mrow) : 1.0f;
+                const float fix = need ? cen - tw : 0.f;
+                if (need) { m_ref = mrow; cen = tw; }
+                {
+                    float l0, l1, t0, t1;
+                    ptx::unpack2(l2, l0, l1);
+                    ptx::unpack2(mt2, t0, t1);
+                    t0 = scale * fmaf(fix, l0, t0);
+                    t1 = scale * fmaf(fix, l1, t1);
+                    l0 *= scale;
+                    l1 *= scale;
+                    l2 = ptx::pack2(l0, l1);
+                    mt2 = ptx::pack2(t0, t1);
+                }
+                if (j > 0) {
+                    // accumulators must be at rest: the value MMAs of tile j-1 have completed
+                    if (!ptx::mbar_wait(bar(C::B_OUTDONE + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    // eight columns at a time: this rare path must not set the register peak of the loop
+                    for (int ch = 2 * sl; ch < 2 * KS; ch += 8) {
 #pragma unroll 1
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t o[8], r[8];
-                        ptx::tmem_ld8(lane_addr + C::COL_ACC0 + 8 * (ch + h), o);
-                        ptx::tmem_ld8(lane_addr + C::COL_ACC1 + 8 * (ch + h), r);
-                        ptx::tmem_wait_ld();
+                        for (int h = 0; h < 2; ++h) {
+                            uint32_t o[8], r[8];
+                            ptx::tmem_ld8(lane_addr + C::COL_ACC0 + 8 * (ch + h), o);
+                            ptx::tmem_ld8(lane_addr + C::COL_ACC1 + 8 * (ch + h), r);
+                            ptx::tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const float ov = __uint_as_float(o[c]);
-                            r[c] = __float_as_uint(scale * fmaf(fix, ov, __uint_as_float(r[c])));
-                            o[c] = __float_as_uint(scale * ov);
+                            for (int c = 0; c < 8; ++c) {
+                                const float ov = __uint_as_float(o[c]);
+                                r[c] = __float_as_uint(scale * fmaf(fix, ov, __uint_as_float(r[c])));
+                                o[c] = __float_as_uint(scale * ov);
+                            }
+                            ptx::tmem_st8(lane_addr + C::COL_ACC0 + 8 * (ch + h), o);
+                            ptx::tmem_st8(lane_addr + C::COL_ACC1 + 8 * (ch + h), r);
                         }
-                        ptx::tmem_st8(lane_addr + C::COL_ACC0 + 8 * (ch + h), o);
-                        ptx::tmem_st8(lane_addr + C::COL_ACC1 + 8 * (ch + h), r);
                     }
                 }
             }
-        }
-        // ---- P~ = 2^(c2 s - m), P~ (T - c); two elements per instruction where the hardware allows
-        const uint64_t nm = ptx::pack2(-m_ref, -m_ref), nc = ptx::pack2(-cen, -cen);
-        uint32_t pp[8], ppt[8];
-#pragma unroll
-        for (int c = 0; c < 16; c += 2) {
-            const uint64_t x2 = ptx::fma2(ptx::pack2u(s[c], s[c + 1]), c2c2, nm);
-            float x0, x1;
-            ptx::unpack2(x2, x0, x1);
-            const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
-            const uint64_t p2 = ptx::pack2(p0, p1);
-            const uint64_t t2 = ptx::fma2(ptx::pack2u(ts[c], ts[c + 1]), aa, nc);
-            const uint64_t pt2 = ptx::mul2(p2, t2);
-            l2 = ptx::add2(l2, p2);
-            mt2 = ptx::add2(mt2, pt2);
-            float q0, q1;
-            ptx::unpack2(pt2, q0, q1);
-            pp[c >> 1] = ptx::pack_bf16(p0, p1);
-            ppt[c >> 1] = ptx::pack_bf16(q0, q1);
-        }
-        // operand of k-step `sl` (16 keys) sits at column 16*sl of the accumulator it replaces
-        ptx::tmem_st8(sbase + 16 * sl, pp);
-        ptx::tmem_st8(sbase + BC + 16 * sl, ppt);
-        ptx::tmem_wait_st();
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
-    }
-
-    if (!ok) break;
-    // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
-    if (item + (int)gridDim.x < items) stage_q(item + gridDim.x);
-    // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R/l - (mu - c) O, lse = ln2 (m + log2 l)
-    if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-    if (ok) {
-        ptx::tc_fence_after_sync();
-        float l0, l1, t0, t1;
-        ptx::unpack2(l2, l0, l1);
-        ptx::unpack2(mt2, t0, t1);
-        xs2[row * 4 + sl] = make_float2(l0 + l1, t0 + t1);
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
-        ok = ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-        ++n_slow;
-    }
-    if (ok) {
-        float l = 0.f, mt = 0.f;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float2 v = xs2[row * 4 + k];
-            l += v.x;
-            mt += v.y;
-        }
-        const float inv = 1.0f / l;
-        const float mun = mt * inv;
-        __nv_bfloat16* o_ptr = p.O + grow * p.d;
-        __nv_bfloat16* t_ptr = p.tO + grow * p.d;
-        for (int ch = sl; ch < KS; ch += 4) {
-            uint32_t o[16], r[16];
-            ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
-            ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, r);
-            ptx::tmem_wait_ld();
-            uint32_t po[8], pt[8];
+            // ---- P~ = 2^(c2 s - m), P~ (T - c); two elements per instruction where the hardware allows
+            const uint64_t nm = ptx::pack2(-m_ref, -m_ref), nc = ptx::pack2(-cen, -cen);
+            uint32_t pp[8], ppt[8];
 #pragma unroll
             for (int c = 0; c < 16; c += 2) {
-                const float o0 = __uint_as_float(o[c]) * inv, o1 = __uint_as_float(o[c + 1]) * inv;
-                const float r0 = fmaf(-mun, o0, __uint_as_float(r[c]) * inv);
-                const float r1 = fmaf(-mun, o1, __uint_as_float(r[c + 1]) * inv);
-                po[c >> 1] = ptx::pack_bf16(o0, o1);
-                pt[c >> 1] = ptx::pack_bf16(r0, r1);
+                const uint64_t x2 = ptx::fma2(ptx::pack2u(s[c], s[c + 1]), c2c2, nm);
+                float x0, x1;
+                ptx::unpack2(x2, x0, x1);
+                const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                const uint64_t p2 = ptx::pack2(p0, p1);
+                const uint64_t t2 = ptx::fma2(ptx::pack2u(ts[c], ts[c + 1]), aa, nc);
+                const uint64_t pt2 = ptx::mul2(p2, t2);
+                l2 = ptx::add2(l2, p2);
+                mt2 = ptx::add2(mt2, pt2);
+                float q0, q1;
+                ptx::unpack2(pt2, q0, q1);
+                pp[c >> 1] = ptx::pack_bf16(p0, p1);
+                ppt[c >> 1] = ptx::pack_bf16(q0, q1);
             }
-            if (row_valid) {
-                *reinterpret_cast<uint4*>(o_ptr + 16 * ch) = make_uint4(po[0], po[1], po[2], po[3]);
-                *reinterpret_cast<uint4*>(t_ptr + 16 * ch) = make_uint4(pt[0], pt[1], pt[2], pt[3]);
-                if (16 * ch + 8 < p.d) {
-                    *reinterpret_cast<uint4*>(o_ptr + 16 * ch + 8) = make_uint4(po[4], po[5], po[6], po[7]);
-                    *reinterpret_cast<uint4*>(t_ptr + 16 * ch + 8) = make_uint4(pt[4], pt[5], pt[6], pt[7]);
+            // operand of k-step `sl` (16 keys) sits at column 16*sl of the accumulator it replaces
+            ptx::tmem_st8(sbase + 16 * sl, pp);
+            ptx::tmem_st8(sbase + BC + 16 * sl, ppt);
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
+        }
+
+        if (!ok) break;
+        // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
+        if (item + (int)gridDim.x < items) stage_q(item + gridDim.x);
+        // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R/l - (mu - c) O, lse = ln2 (m + log2 l)
+        if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            float l0, l1, t0, t1;
+            ptx::unpack2(l2, l0, l1);
+            ptx::unpack2(mt2, t0, t1);
+            xs2[row * 4 + sl] = make_float2(l0 + l1, t0 + t1);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
+            ok = ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            ++n_slow;
+        }
+        if (ok) {
+            float l = 0.f, mt = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 v = xs2[row * 4 + k];
+                l += v.x;
+                mt += v.y;
+            }
+            const float inv = 1.0f / l;
+            const float mun = mt * inv;
+            __nv_bfloat16* o_ptr = p.O + grow * p.d;
+            __nv_bfloat16* t_ptr = p.tO + grow * p.d;
+            for (int ch = sl; ch < KS; ch += 4) {
+                uint32_t o[16], r[16];
+                ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
+                ptx::tmem_ld16(lane_addr + C::COL_ACC1 + 16 * ch, r);
+                ptx::tmem_wait_ld();
+                uint32_t po[8], pt[8];
+#pragma unroll
+                for (int c = 0; c < 16; c += 2) {
+                    const float o0 = __uint_as_float(o[c]) * inv, o1 = __uint_as_float(o[c + 1]) * inv;
+                    const float r0 = fmaf(-mun, o0, __uint_as_float(r[c]) * inv);
+                    const float r1 = fmaf(-mun, o1, __uint_as_float(r[c + 1]) * inv);
+                    po[c >> 1] = ptx::pack_bf16(o0, o1);
+                    pt[c >> 1] = ptx::pack_bf16(r0, r1);
+                }
+                if (row_valid) {
+                    *reinterpret_cast<uint4*>(o_ptr + 16 * ch) = make_uint4(po[0], po[1], po[2], po[3]);
+                    *reinterpret_cast<uint4*>(t_ptr + 16 * ch) = make_uint4(pt[0], pt[1], pt[2], pt[3]);
+                    if (16 * ch + 8 < p.d) {
+                        *reinterpret_cast<uint4*>(o_ptr + 16 * ch + 8) = make_uint4(po[4], po[5], po[6], po[7]);
+                        *reinterpret_cast<uint4*>(t_ptr + 16 * ch + 8) = make_uint4(pt[4], pt[5], pt[6], pt[7]);
+                    }
                 }
             }
+            if (sl == 0 && row_valid) {
+                p.lse[grow] = (m_ref + log2f(l)) * 0.6931471805599453f;
+                p.mu[grow] = cen + mun;
+            }
         }
-        if (sl == 0 && row_valid) {
-            p.lse[grow] = (m_ref + log2f(l)) * 0.6931471805599453f;
-            p.mu[grow] = cen + mun;
-        }
-    }
     }
 }
 
@@ -513,38 +513,38 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         bool ok = true;
         int g = 0, it = 0;
         for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
-        // Q, tQ of this item are in tensor memory (the element-wise warps stage them as soon as they have
-        // seen the last scores of the item before)
-        ok = ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-        for (int j = 0; ok && j < T; ++j, ++g) {
-            const int b = g & 1;
-            ok = ptx::mbar_wait_warp(bar(C::B_EFULL + g % SE), (g / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            // the score buffer is free once the value MMAs of tile g-2 have read their operands out of it
-            if (ok && g >= 2) ok = ptx::mbar_wait_warp(bar(C::B_OUTDONE + b), ((g - 2) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, g), 16, 1024);
-            const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, g), 16, 1024);
-            const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
+            // Q, tQ of this item are in tensor memory (the element-wise warps stage them as soon as they have
+            // seen the last scores of the item before)
+            ok = ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+            for (int j = 0; ok && j < T; ++j, ++g) {
+                const int b = g & 1;
+                ok = ptx::mbar_wait_warp(bar(C::B_EFULL + g % SE), (g / SE) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+                // the score buffer is free once the value MMAs of tile g-2 have read their operands out of it
+                if (ok && g >= 2) ok = ptx::mbar_wait_warp(bar(C::B_OUTDONE + b), ((g - 2) >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint64_t kd = ptx::smem_desc_sw128(tile_addr(0, g), 16, 1024);
+                const uint64_t tkd = ptx::smem_desc_sw128(tile_addr(1, g), 16, 1024);
+                const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {  // S = Q K^T
-                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                ptx::mma_ts_elect(dS, aq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
-            }
-            ptx::mma_commit_elect(bar(C::B_SFULL + b));
+                for (int kk = 0; kk < KS; ++kk) {  // S = Q K^T
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dS, aq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
+                }
+                ptx::mma_commit_elect(bar(C::B_SFULL + b));
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {  // Sd = tQ K^T
-                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                ptx::mma_ts_elect(dT, atq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
-            }
+                for (int kk = 0; kk < KS; ++kk) {  // Sd = tQ K^T
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dT, atq + 8 * kk, kd + off, idesc_s, kk > 0 ? 1u : 0u);
+                }
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {  // Sd += Q tK^T
-                const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
+                for (int kk = 0; kk < KS; ++kk) {  // Sd += Q tK^T
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                    ptx::mma_ts_elect(dT, aq + 8 * kk, tkd + off, idesc_s, 1u);
+                }
+                ptx::mma_commit_elect(bar(C::B_SFULL + 2 + b));
+                ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
             }
-            ptx::mma_commit_elect(bar(C::B_SFULL + 2 + b));
-            ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
-        }
         }
     } else if (warp == 3) {
         constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
@@ -553,31 +553,31 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         bool ok = true;
         int g = 0;
         for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
-        // The first tile of an item overwrites the accumulators (accumulate = 0): every element-wise warp
-        // reads them out for the item before (its epilogue) before it turns to this tile, whose operands
-        // the wait below is for.
-        for (int j = 0; ok && j < T; ++j, ++g) {
-            const int b = g & 1;
-            ok = ptx::mbar_wait_warp(bar(C::B_LFULL + g % SL), (g / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            if (ok) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
-            // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
-            const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);
-            const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
+            // The first tile of an item overwrites the accumulators (accumulate = 0): every element-wise warp
+            // reads them out for the item before (its epilogue) before it turns to this tile, whose operands
+            // the wait below is for.
+            for (int j = 0; ok && j < T; ++j, ++g) {
+                const int b = g & 1;
+                ok = ptx::mbar_wait_warp(bar(C::B_LFULL + g % SL), (g / SL) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+                if (ok) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + b), (g >> 1) & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
+                // MN-major B: atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
+                const uint64_t vd = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);
+                const uint64_t tvd = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
 #pragma unroll
-            for (int u = 0; u < BC / 16; ++u) {
-                const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
-                const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                ptx::mma_ts_elect(acc0, a0 + 16 * u, vd + off, idesc_o, acc);   // O~ += P~ V
-                ptx::mma_ts_elect(acc1, a1 + 16 * u, vd + off, idesc_o, acc);   // R  += P~(T-c) V
-                ptx::mma_ts_elect(acc1, a0 + 16 * u, tvd + off, idesc_o, 1u);   // R  += P~ tV
+                for (int u = 0; u < BC / 16; ++u) {
+                    const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                    const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                    ptx::mma_ts_elect(acc0, a0 + 16 * u, vd + off, idesc_o, acc);   // O~ += P~ V
+                    ptx::mma_ts_elect(acc1, a1 + 16 * u, vd + off, idesc_o, acc);   // R  += P~(T-c) V
+                    ptx::mma_ts_elect(acc1, a0 + 16 * u, tvd + off, idesc_o, 1u);   // R  += P~ tV
+                }
+                ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
+                ptx::mma_commit_elect(bar(C::B_OUTDONE + b));
+                if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
             }
-            ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
-            ptx::mma_commit_elect(bar(C::B_OUTDONE + b));
-            if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
-        }
         }
     } else if (warp >= 4) {
         fwd_elementwise<DP>(p, tmem_base, bar0, abort_flag, xmax, xslow, warp - 4, lane, items, row_tiles, T);
