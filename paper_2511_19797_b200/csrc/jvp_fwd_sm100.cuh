@@ -94,7 +94,7 @@ struct FwdCfg {
     static constexpr int NBARS = B_XSLOW + 4;
     static_assert(NBARS <= 48, "barrier table too small");
     static constexpr int XMAX_FLOATS = 2 * 128 * 4;   // [parity][row][slice]
-    static constexpr int XSLOW_FLOATS = 128 * 4 * 2;  // [row][slice][2]
+    static constexpr int XSLOW_FLOATS = 2 * 128 * 4 * 2;  // [exchange parity][row][slice][2]
     static constexpr int MISC_BYTES = 48 * 8 + 64 + (XMAX_FLOATS + XSLOW_FLOATS) * 4;
     static constexpr int SMEM_BYTES = TILE_BYTES + MISC_BYTES + 1024 /*alignment slack*/;
     // TMEM columns: accumulators O~ and R, the bf16 operands Q and tQ in the gaps behind them, and
@@ -205,7 +205,8 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
                     la = gt ? __uint_as_float(s[c]) : la;
                     lt = gt ? __uint_as_float(ts[c]) : lt;
                 }
-                xs2[row * 4 + sl] = make_float2(la, lt);
+                float2* xb = xs2 + (n_slow & 1) * 512;  // consecutive exchanges use different halves
+                xb[row * 4 + sl] = make_float2(la, lt);
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
                 if (!ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS)) { ok = false; break; }
@@ -213,7 +214,7 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
                 float ba = -CUDART_INF_F, bt = 0.f;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {  // ties go to the lowest slice
-                    const float2 v = xs2[row * 4 + k];
+                    const float2 v = xb[row * 4 + k];
                     const bool gt = v.x > ba;
                     ba = gt ? v.x : ba;
                     bt = gt ? v.y : bt;
@@ -286,26 +287,64 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
         }
 
         if (!ok) break;
-        // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
-        if (item + (int)gridDim.x < items) stage_q(item + gridDim.x);
+        // The next item's operands, so that its loads and first score MMAs run under this item's epilogue.  Their
+        // global loads are issued first and land while the row sums are exchanged (which needs no MMA result).
+        const bool has_next = item + (int)gridDim.x < items;
+        constexpr int NCH = (2 * KS + 3) / 4;  // chunks of 16 columns per warp, at most
+        uint4 nq[NCH][2];
+        {
+            const int nitem = has_next ? item + (int)gridDim.x : item;
+            const int bh_ = nitem / row_tiles;
+            const int row0_ = (nitem - bh_ * row_tiles) * FWD_ROWS;
+            const bool valid_ = has_next && row0_ + row < p.N;
+            const size_t grow_ = (size_t)bh_ * p.N + row0_ + row;
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) {
+                const int ch = sl + 4 * i;
+                const bool is_t = ch >= KS;
+                const int kk = is_t ? ch - KS : ch;
+                const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow_ * p.d + 16 * kk;
+                nq[i][0] = nq[i][1] = make_uint4(0, 0, 0, 0);
+                if (ch < 2 * KS && valid_ && 16 * kk < p.d) nq[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
+                if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) nq[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
+            }
+        }
         // ---- epilogue: O = O~/l, mu - c = mt/l, tO = R/l - (mu - c) O, lse = ln2 (m + log2 l)
-        if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
-        if (ok) {
-            ptx::tc_fence_after_sync();
+        float2* xe;
+        {
             float l0, l1, t0, t1;
             ptx::unpack2(l2, l0, l1);
             ptx::unpack2(mt2, t0, t1);
-            xs2[row * 4 + sl] = make_float2(l0 + l1, t0 + t1);
+            xe = xs2 + (n_slow & 1) * 512;
+            xe[row * 4 + sl] = make_float2(l0 + l1, t0 + t1);
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(C::B_XSLOW + q));
             ok = ptx::mbar_wait(bar(C::B_XSLOW + q), n_slow & 1, abort_flag, FWD_WAIT_LIMIT_NS);
             ++n_slow;
         }
+        if (has_next) {
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) {
+                const int ch = sl + 4 * i;
+                if (ch < 2 * KS) {
+                    const bool is_t = ch >= KS;
+                    const int kk = is_t ? ch - KS : ch;
+                    const uint32_t r[8] = {nq[i][0].x, nq[i][0].y, nq[i][0].z, nq[i][0].w, nq[i][1].x, nq[i][1].y, nq[i][1].z, nq[i][1].w};
+                    ptx::tmem_st8(lane_addr + (is_t ? C::COL_TQ : C::COL_Q) + 8 * kk, r);
+                }
+            }
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+        }
+        if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, FWD_WAIT_LIMIT_NS);
+        if (ok) ptx::tc_fence_after_sync();
         if (ok) {
             float l = 0.f, mt = 0.f;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float2 v = xs2[row * 4 + k];
+                const float2 v = xe[row * 4 + k];
                 l += v.x;
                 mt += v.y;
             }
