@@ -239,7 +239,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             if (C::TRANSPOSED)
                 if (!ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after_sync();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 0);
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 0);
             const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
             const int key0 = j * BC + 16 * sl;  // first stream row of this slice
             if (NPAIR == 1) {
@@ -323,15 +323,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     }
                 }
                 // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 2);
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 2);
                 if (!ptx::mbar_wait(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 3);
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 3);
                 uint32_t s3[16], s4[16];
                 ptx::tmem_ld16(sbase + 2 * BC, s3);
                 ptx::tmem_ld16(sbase + 3 * BC, s4);
                 ptx::tmem_wait_ld();
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 4);
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 4);
                 uint32_t pa0[8], pa1[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
@@ -344,19 +344,20 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     pa0[k] = ptx::pack_bf16(w0, w1);
                     pa1[k] = ptx::pack_bf16(d0, d1);
                 }
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 5);
+                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 5);
                 ptx::tmem_st8(sbase + 2 * BC, pa0);
                 ptx::tmem_st8(sbase + 3 * BC, pa1);
             }
             ptx::tmem_wait_st();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 6);
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 6);
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, j, 1);
-            if (lane == 0) BTL_STAMP(4 + (w >> 3), j, w & 7);
+            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 1);
+            if (lane == 0) BTL_STAMP(4 + (w >> 3), g, w & 7);
             if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
         }
         if (!ok) break;
+        if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 0);  // tiles of the item done (warp 0)
         // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
         if (item + (int)gridDim.x < items) {
             if (NPAIR == 1) {
@@ -367,7 +368,9 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             }
             stage_x(item + gridDim.x);
         }
+        if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 2);  // next item's operands staged (warp 0)
         if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+        if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 3);  // last output MMAs of the item done
         if (ok) {
             ptx::tc_fence_after_sync();
             __nv_bfloat16* p0 = p.out0 + grow * p.d;
@@ -392,7 +395,8 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     }
                 }
             }
-            // the accumulators may be overwritten by the first output MMAs of the next item
+            if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 1);  // epilogue of the item done (warp 0)
+        // the accumulators may be overwritten by the first output MMAs of the next item
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(C::B_ACCFREE));
@@ -756,12 +760,23 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // The turn passes on after the whole batch (outputs(g), S(g + 2)): two batches queued at once
             // would share the pipe MMA by MMA, both would finish late and together, and the element-wise
             // work of the two buffers would then run back to back instead of under the other's MMAs.
+            // Where the score MMAs belong to the next item they wait for its operands, which the element-wise
+            // warps stage after their last tile: there the turn passes on before them, or the last output MMAs of
+            // this item, and with them its epilogue, would wait for the next item's operands too.
             for (int g = wsel; ok && g < G; g += 2) {
                 ok = issue_outputs(g);  // waits for the L tile, the operands and its turn
+                const bool cross = g % T + 2 >= T;
+                if (cross) {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)g + 1u);
+                }
                 if (ok && g + 2 < G) ok = issue_scores(g + 2);
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)g + 1u);
+                if (!cross) {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)g + 1u);
+                }
             }
         } else {
             if (wsel == 0) {  // one issuer: splitting these steps over two warps measured 1 to 2 % slower
