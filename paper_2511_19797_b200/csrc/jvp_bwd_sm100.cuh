@@ -124,10 +124,13 @@ struct BwdCfg {
     static constexpr int B_SFULL = B_LEMPTY + SL;          // DV: per buffer.  DK/DQ: +0 (S, Sd) written, +1 (D, X) written
     static constexpr int B_PREADY = B_SFULL + 2;           // DV: per buffer.  DK/DQ: +0 operands written, +1 (S, Sd) read
     static constexpr int B_FINAL = B_PREADY + 2;
-    static constexpr int B_QREADY = B_FINAL + 1;
-    static constexpr int B_OWNER = B_QREADY + 1;
-    static constexpr int B_ACCFREE = B_OWNER + 1;  // the element-wise warps have read the accumulators of an item
-    static constexpr int B_OWNFREE = B_ACCFREE + 1;  // the MMAs that read the shared-memory owner tiles of an item are done
+    // Per-item barriers that the two alternating DV issuers wait on come in pairs, one for even and one for odd
+    // items of the CTA: with an odd number of tiles per item (or one) an issuer meets only every other item, and
+    // a parity wait on a single barrier would then take the completion of the item before last for its own.
+    static constexpr int B_QREADY = B_FINAL + 1;   // + (item & 1): the owner operands of the item are in tensor memory
+    static constexpr int B_OWNER = B_QREADY + 2;
+    static constexpr int B_ACCFREE = B_OWNER + 1;  // + (item & 1): the element-wise warps have read the item's accumulators
+    static constexpr int B_OWNFREE = B_ACCFREE + 2;  // the MMAs that read the shared-memory owner tiles of an item are done
     static constexpr int NBARS = B_OWNFREE + 1;
     static_assert(NBARS <= 48, "barrier table too small");
     static constexpr int STATS_FLOATS = SL * 4 * 64;
@@ -180,7 +183,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     // ---- owner rows of X0 and X1 of an item -> bf16 operands in tensor memory (k-step kk at 8 packed
     // columns); all of this warp's loads first, then the stores: one global-memory latency instead of one
     // per chunk.  Called once no MMA reads the operands of the item before any more.
-    auto stage_x = [&](int item) {
+    auto stage_x = [&](int item, int item_index) {
         const int bh_ = item / row_tiles;
         const int row0_ = (item - bh_ * row_tiles) * BWD_ROWS;
         const bool valid_ = row0_ + row < p.N;
@@ -210,12 +213,12 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY));
+        if (lane == 0) ptx::mbar_arrive(bar(C::B_QREADY + (item_index & 1)));
     };
 
     bool ok = true;
     int it = 0;  // items done by this CTA
-    if ((int)blockIdx.x < items) stage_x(blockIdx.x);
+    if ((int)blockIdx.x < items) stage_x(blockIdx.x, 0);
     for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
         const int g0 = it * T;  // tiles this CTA has streamed before this item: rings and barrier phases run on
         const int bh = item / row_tiles;
@@ -366,7 +369,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 const int gl = g0 + T - 1;
                 if (!ptx::mbar_wait(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             }
-            stage_x(item + gridDim.x);
+            stage_x(item + gridDim.x, it + 1);
         }
         if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 2);  // next item's operands staged (warp 0)
         if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
@@ -399,7 +402,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         // the accumulators may be overwritten by the first output MMAs of the next item
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(C::B_ACCFREE));
+            if (lane == 0) ptx::mbar_arrive(bar(C::B_ACCFREE + (it & 1)));
         }
     }
 }
@@ -449,8 +452,10 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         }
         ptx::mbar_init(bar(C::B_FINAL), 1);
         ptx::mbar_init(bar(C::B_QREADY), 16);
+        ptx::mbar_init(bar(C::B_QREADY + 1), 16);
         ptx::mbar_init(bar(C::B_OWNER), C::FULL_COUNT);
         ptx::mbar_init(bar(C::B_ACCFREE), 16);
+        ptx::mbar_init(bar(C::B_ACCFREE + 1), 16);
         ptx::mbar_init(bar(C::B_OWNFREE), 1);
         ptx::fence_mbar_init();
     }
@@ -548,6 +553,10 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                 __syncwarp();
                                 if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
                                 pend_s = -1;
+                                if (owner_pend) {  // an item of one tile: its owner copies were not signalled yet either
+                                    if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
+                                    owner_pend = false;
+                                }
                             }
                         }
                         ok = ptx::mbar_wait_warp(bar(C::B_OWNFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
@@ -704,7 +713,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const int b = g & 1, it = g / T, j = g - it * T;
             if (!ptx::mbar_wait_warp(bar(C::B_EFULL + g % SE), (g / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             // the first tiles of an item: its owner operands are in tensor memory
-            if (j < 2 && !ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (j < 2 && !ptx::mbar_wait_warp(bar(C::B_QREADY + (it & 1)), (it >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
             if (lane == 0) BTL_STAMP(0, g, 0);
             // Y0, Y1 in the E ring, K-major B
@@ -732,7 +741,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // the other issuer has queued its batch of tile g - 1: accumulation order is the tile order
             if (!ptx::turn_wait_warp(turn_addr, (uint32_t)g, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             // the first tile of an item overwrites the accumulators: all sixteen element-wise warps have read them
-            if (j == 0 && it > 0 && !ptx::mbar_wait_warp(bar(C::B_ACCFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
+            if (j == 0 && it > 0 && !ptx::mbar_wait_warp(bar(C::B_ACCFREE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
             if (lane == 0) BTL_STAMP(0, g, 3);
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
@@ -820,7 +829,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int g0 = it * T;
                     // the item's owner operands: X0, X1 in tensor memory, X2, X3 in shared memory
-                    ok = ptx::mbar_wait_warp(bar(C::B_QREADY), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                    ok = ptx::mbar_wait_warp(bar(C::B_QREADY + (it & 1)), (it >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     if (ok) ok = ptx::mbar_wait_warp(bar(C::B_OWNER), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     // (S, Sd) of the tile before, the last of the item before, read by all element-wise warps
                     if (ok && it > 0) ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 1), (g0 - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
@@ -852,7 +861,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         if (lane == 0) BTL_STAMP(0, g, 2);
                         ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), g & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                         // the first tile of an item overwrites the accumulators: the element-wise warps have read them
-                        if (ok && j == 0 && it > 0) ok = ptx::mbar_wait_warp(bar(C::B_ACCFREE), (it - 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                        if (ok && j == 0 && it > 0) ok = ptx::mbar_wait_warp(bar(C::B_ACCFREE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
                         if (lane == 0) BTL_STAMP(0, g, 3);

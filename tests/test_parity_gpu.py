@@ -61,11 +61,12 @@ def test_ragged_and_degenerate_shapes(B, H, N, d, mode):
         assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
 
 
-@pytest.mark.parametrize("B,H,N,d", [(3, 50, 192, 72), (3, 50, 320, 64), (5, 61, 65, 72), (2, 80, 200, 40)])
+@pytest.mark.parametrize("B,H,N,d", [(3, 50, 192, 72), (3, 50, 320, 64), (5, 61, 65, 72), (2, 80, 200, 40),
+                                     (4, 50, 64, 72), (4, 50, 33, 40)])
 def test_several_work_items_per_cta(B, H, N, d):
     """More work items than SMs (one CTA per SM walks through several of them), with odd numbers of stream
-    tiles per item (3, 5, 2, 4 tiles of 64), so that buffer and barrier parities differ from item to item, and
-    a ragged last tile."""
+    tiles per item (3, 5, 2, 4, 1, 1 tiles of 64), so that buffer and barrier parities differ from item to item,
+    and a ragged last tile."""
     wl = inputs.custom(B, H, N, d, seed=300 + N + d)
     errs, _, _ = run_case(wl)
     assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
