@@ -72,6 +72,19 @@ def test_several_work_items_per_cta(B, H, N, d):
     assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
 
 
+@pytest.mark.parametrize("B,H,N,d", [
+    (1, 108, 129, 80), (1, 173, 383, 72), (1, 559, 16, 8), (2, 17, 640, 40), (2, 210, 65, 72), (2, 95, 383, 64),
+    (3, 116, 65, 80), (3, 43, 384, 80), (3, 27, 640, 64), (5, 102, 31, 56), (5, 16, 250, 48), (5, 40, 128, 64),
+])
+def test_many_heads_of_odd_shapes_on_sampled_heads(B, H, N, d):
+    """Shapes drawn at random (sequence lengths around the tile boundaries, every padded head dim), each with
+    more work items than SMs; the oracle runs on a dozen sampled heads."""
+    wl = inputs.custom(B, H, N, d, seed=1000 + N + d)
+    heads = sorted(set(int(i) for i in np.random.default_rng(N * 131 + d).integers(0, B * H, 12)))
+    errs, _, _ = run_case(wl, oracle_heads=heads)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
 def test_explicit_scale_is_honoured():
     wl = inputs.custom(1, 2, 96, 48, seed=7)
     errs, _, _ = run_case(wl, scale=0.05)
