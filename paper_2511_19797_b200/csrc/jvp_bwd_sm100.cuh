@@ -709,8 +709,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         // tiles this CTA streams over all of its items; tile g belongs to item g / T of this CTA
         const int n_it = (int)blockIdx.x < items ? (items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
         const int G = n_it * T;
-        auto issue_scores = [&](int g) -> bool {  // DV only (the two-pair passes have their own loop below)
-            const int b = g & 1, it = g / T, j = g - it * T;
+        // (it, j): item of this CTA and tile inside it, g = it * T + j (kept by the caller: no division per tile)
+        auto issue_scores = [&](int g, int it, int j) -> bool {  // DV only (the two-pair passes have their own loop below)
+            const int b = g & 1;
             if (!ptx::mbar_wait_warp(bar(C::B_EFULL + g % SE), (g / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             // the first tiles of an item: its owner operands are in tensor memory
             if (j < 2 && !ptx::mbar_wait_warp(bar(C::B_QREADY + (it & 1)), (it >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
@@ -733,8 +734,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             if (lane == 0) BTL_STAMP(0, g, 1);
             return true;
         };
-        auto issue_outputs = [&](int g) -> bool {  // DV only
-            const int b = g & 1, it = g / T, j = g - it * T;
+        auto issue_outputs = [&](int g, int it, int j) -> bool {  // DV only
+            const int b = g & 1;
             if (lane == 0) BTL_STAMP(0, g, 2);
             if (!ptx::mbar_wait_warp(bar(C::B_LFULL + g % SL), (g / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (g >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
@@ -765,7 +766,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         bool ok = true;
         if constexpr (NPAIR == 1) {
             // warp `wsel` owns the tiles g = wsel, wsel + 2, ...: S(g), then per tile outputs(g) and S(g + 2)
-            if (wsel < G) ok = issue_scores(wsel);
+            int it = 0, j = wsel;  // of tile g
+            while (j >= T) { j -= T; ++it; }
+            if (wsel < G) ok = issue_scores(wsel, it, j);
             // The turn passes on after the whole batch (outputs(g), S(g + 2)): two batches queued at once
             // would share the pipe MMA by MMA, both would finish late and together, and the element-wise
             // work of the two buffers would then run back to back instead of under the other's MMAs.
@@ -773,14 +776,16 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // warps stage after their last tile: there the turn passes on before them, or the last output MMAs of
             // this item, and with them its epilogue, would wait for the next item's operands too.
             for (int g = wsel; ok && g < G; g += 2) {
-                ok = issue_outputs(g);  // waits for the L tile, the operands and its turn
-                const bool cross = g % T + 2 >= T;
+                ok = issue_outputs(g, it, j);  // waits for the L tile, the operands and its turn
+                const bool cross = j + 2 >= T;
                 if (cross) {
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::turn_post(turn_addr, (uint32_t)g + 1u);
                 }
-                if (ok && g + 2 < G) ok = issue_scores(g + 2);
+                j += 2;
+                while (j >= T) { j -= T; ++it; }
+                if (ok && g + 2 < G) ok = issue_scores(g + 2, it, j);
                 if (!cross) {
                     ptx::tc_fence_before_sync();
                     __syncwarp();
