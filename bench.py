@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 KERNEL_GEMMS = {"fwd": 6, "bwd_rowsums": 0, "bwd_dv": 6, "bwd_dk": 9, "bwd_dq": 9}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
 # profiles/jvp_fwd_bwd_kernels_dit512.md (that workload only; None for anything else)
-NCU_TRAFFIC_BYTES = {"dit512": {"fwd": 281.5e6, "bwd_dv": 282.0e6, "bwd_dk": 364.5e6, "bwd_dq": 363.7e6}}
+NCU_TRAFFIC_BYTES = {"dit512": {"fwd": 282.4e6, "bwd_dv": 280.7e6, "bwd_dk": 364.2e6, "bwd_dq": 364.1e6}}
 
 
 def load_peaks():
