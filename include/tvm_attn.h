@@ -15,7 +15,11 @@
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
  *     and the call returns without synchronising.
  *   - Return value: TVM_ATTN_OK or a negative tvm_attn_status.  No exception or abort crosses
- *     this boundary.  Concurrent calls from several host threads on different streams are allowed.
+ *     this boundary.  Concurrent calls from several host threads on different streams are allowed
+ *     (each call with its own workspace); the per-kernel timing aid below is the exception and is to
+ *     be driven from one thread while it is enabled.
+ *   - After a call returns, its results are complete for any work enqueued later on the same stream
+ *     (plain stream order), although the kernels of one backward call overlap one another.
  *   - Self-attention, non-causal, no mask, bias or dropout: N queries attend to N keys per head.
  */
 #ifndef TVM_ATTN_H_
@@ -115,7 +119,9 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
  *     library holds it until the process exits, whether or not this function is ever called.
  *   - It calls neither cudaMalloc nor cudaFree nor any allocating library routine.
  *   - The first call on each device looks up the array's device address (once per device, with that
- *     device current).  Make that first call outside any stream capture.
+ *     device current) and keeps it for the life of the process.  Make that first call outside any
+ *     stream capture.  Devices with index 0..63 are supported (TVM_ATTN_CUDA_ERROR beyond), and the
+ *     kept address does not survive a cudaDeviceReset of that device.
  *   - All calls on a device share the one array.  Nothing in it has to start at zero (the pass rewrites
  *     all of it before reading it) and its contents after a call are unspecified.  Two calls that may
  *     run at the same time on the GPU (different streams, different host threads) race on it: serialise
@@ -132,8 +138,21 @@ int tvm_attn_jvp_bwd_noalloc(const tvm_attn_params* p, const void* Q, const void
  * recorded: TVM_ATTN_OK, TVM_ATTN_DEVICE_TIMEOUT if a bounded wait inside a tensor-core kernel gave
  * up (its outputs are then unspecified; the context stays usable), or TVM_ATTN_CUDA_ERROR.  Clears
  * the recorded status.  (No counterpart in the paper: error reporting of this library.)
+ * The status is one word per device, not per stream: tensor-core kernels that start while it is raised
+ * return at once without touching their outputs, and with several host threads the time-out reported
+ * to one of them may have been raised by another thread's call.
  */
 int tvm_attn_check_status(void* cuda_stream);
+
+/*
+ * Exercises the time-out reporting without disturbing a real kernel (no counterpart in the paper).
+ * Enqueues a one-warp kernel that waits on a barrier nobody signals, with the same bounded wait the
+ * tensor-core kernels use, and gives up after `limit_ns` nanoseconds (1 .. 100,000,000; a millisecond
+ * is plenty).  It then raises the device status exactly like a kernel whose wait ran out: the next
+ * tvm_attn_check_status returns TVM_ATTN_DEVICE_TIMEOUT, and tensor-core kernels enqueued in between
+ * are no-ops.  Nothing hangs and the context stays usable.
+ */
+int tvm_attn_selftest_timeout(uint64_t limit_ns, void* cuda_stream);
 
 /*
  * Per-kernel timing aid (no counterpart in the paper).  While enabled, tvm_attn_jvp_fwd/bwd record

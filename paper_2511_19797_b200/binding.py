@@ -33,7 +33,7 @@ class Params(ctypes.Structure):
 
 _lib = None
 EXPORTS = ("tvm_attn_jvp_workspace_bytes", "tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_jvp_bwd_noalloc",
-           "tvm_attn_check_status",
+           "tvm_attn_check_status", "tvm_attn_selftest_timeout",
            "tvm_attn_launch_count", "tvm_attn_strerror", "tvm_attn_version", "tvm_attn_set_profiling",
            "tvm_attn_get_profile")
 
@@ -65,6 +65,8 @@ def load(build_if_missing=False):
     lib.tvm_attn_jvp_bwd_noalloc.argtypes = [pp] + [vp] * 18 + [vp]
     lib.tvm_attn_check_status.restype = ctypes.c_int
     lib.tvm_attn_check_status.argtypes = [vp]
+    lib.tvm_attn_selftest_timeout.restype = ctypes.c_int
+    lib.tvm_attn_selftest_timeout.argtypes = [ctypes.c_uint64, vp]
     lib.tvm_attn_launch_count.restype = ctypes.c_uint64
     lib.tvm_attn_launch_count.argtypes = []
     lib.tvm_attn_strerror.restype = ctypes.c_char_p
@@ -179,6 +181,13 @@ def tvm_attn_check_status(stream=None, raise_on_error=True):
     if rc != 0 and raise_on_error:
         _raise("tvm_attn_check_status", rc)
     return rc
+
+
+def tvm_attn_selftest_timeout(limit_ns=1_000_000, stream=None):
+    """Enqueues the kernel whose bounded wait runs out on purpose (see include/tvm_attn.h)."""
+    rc = int(load().tvm_attn_selftest_timeout(int(limit_ns), _stream_ptr(stream)))
+    if rc != 0:
+        _raise("tvm_attn_selftest_timeout", rc)
 
 
 def tvm_attn_launch_count():

@@ -25,15 +25,15 @@ def nvcc_command(out_path, extra=()):
             *extra, "-o", out_path, *[os.path.join(CSRC, s) for s in SOURCES]]
 
 
-def build(force=False, verbose=False, out_path=None, defines=()):
+def build(force=False, verbose=False, out_path=None):
     """Compiles libtvm_attn.so if it is missing or older than its sources; returns its path.
-    `out_path` and `defines` (e.g. ("TVM_ATTN_DEBUG_DUMP",)) make a separate, differently configured copy."""
+    `out_path` writes the library somewhere else."""
     global_out = out_path or LIB_PATH
     if not force and os.path.exists(global_out) and os.path.getmtime(global_out) >= _newest_source_mtime():
         return global_out
     os.makedirs(os.path.dirname(global_out), exist_ok=True)
     tmp = global_out + ".tmp.%d" % os.getpid()
-    extra = tuple("-D" + d for d in defines) + (("-Xptxas", "-v") if verbose else ())
+    extra = ("-Xptxas", "-v") if verbose else ()
     cmd = nvcc_command(tmp, extra)
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:

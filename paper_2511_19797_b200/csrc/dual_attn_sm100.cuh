@@ -61,7 +61,6 @@ struct TcParams {
     const float* sig1;
     const float* cvec;
     int* status;      // device status word; non-zero makes the kernel a no-op
-    float* dbg;       // debug builds only: receives the raw score accumulators of the first tile of CTA 0
 };
 
 template <int MODE, int NA>
@@ -351,14 +350,6 @@ dual_attn_kernel(const __grid_constant__ CUtensorMap tm_own0, const __grid_const
                 ptx::tmem_ld16(sbase + BC + col0, ts);
                 ptx::tmem_ld16(sbase + BC + col0 + 16, ts + 16);
                 ptx::tmem_wait_ld();
-#ifdef TVM_ATTN_DEBUG_DUMP
-                if (p.dbg && blockIdx.x == 0 && j == 0) {
-                    for (int c = 0; c < 32; ++c) {
-                        p.dbg[row * 64 + col0 + c] = __uint_as_float(s[c]);
-                        p.dbg[128 * 64 + row * 64 + col0 + c] = __uint_as_float(ts[c]);
-                    }
-                }
-#endif
                 const int nvalid = p.N - j * BC - col0;  // columns of this half that are real keys
                 if (nvalid < 32) {
 #pragma unroll

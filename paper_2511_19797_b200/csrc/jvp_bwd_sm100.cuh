@@ -69,24 +69,7 @@ struct BwdParams {
     const float* sig1;  // rowsum(dtO * O)
     const float* cvec;  // rowsum(dO * O) + rowsum(dtO * tO)
     int* status;        // device status word; non-zero makes the kernel a no-op
-    unsigned long long* tl;  // timeline builds only: clock stamps of one CTA
 };
-
-#ifdef TVM_ATTN_TIMELINE
-#ifndef TVM_ATTN_TIMELINE_CTA
-#define TVM_ATTN_TIMELINE_CTA 0  // the CTA whose clock stamps are recorded
-#endif
-#define BTL_STAMP(role, j, ev)                                                                         \
-    do {                                                                                                \
-        if (p.tl && blockIdx.x == TVM_ATTN_TIMELINE_CTA && (j) < 64) {                            \
-            unsigned long long t_;                                                                      \
-            asm volatile("mov.u64 %0, %clock64;" : "=l"(t_));                                          \
-            p.tl[((role) * 64 + (j)) * 8 + (ev)] = t_;                                                  \
-        }                                                                                               \
-    } while (0)
-#else
-#define BTL_STAMP(role, j, ev) do {} while (0)
-#endif
 
 template <int MODE, int DP>
 struct BwdCfg {
@@ -103,6 +86,12 @@ struct BwdCfg {
     // single N = DP operand needs one layout: two 128-byte-swizzled atoms.
     static constexpr int OWN_BYTES = BWD_ROWS * 128 + (NA - 1) * BWD_ROWS * 32;  // one owner tensor in shared memory
     static constexpr int NOWN_SMEM = NPAIR == 2 ? 2 : 0;
+    // DK, DQ: which owner pair lives in tensor memory.  The second score pair sits on the critical path of a tile
+    // (second pair -> element-wise phase B -> output MMAs -> second pair of the next tile) while the first pair
+    // runs under it, so the second pair gets the tensor-memory operands (full MMA rate) and the first pair reads
+    // its A operands from shared memory (bound by the shared-memory port, but hidden).
+    static constexpr int XT0 = NPAIR == 2 ? 2 : 0;  // p.own[XT0], p.own[XT0 + 1] -> tensor memory
+    static constexpr int XS0 = NPAIR == 2 ? 0 : 2;  // p.own[XS0], p.own[XS0 + 1] -> shared memory (two-pair passes)
     static constexpr int EST_BYTES = BC * 128 + (NA - 1) * BC * 32;  // one E-ring tile
     static constexpr int LST_BYTES = NA * BC * 128;                  // one L-ring tile
     static constexpr int SE = NPAIR == 1 ? 4 : (NA == 1 ? 4 : 3);
@@ -195,7 +184,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             const int ch = slot + 4 * i;
             const bool second = ch >= KS;
             const int kk = second ? ch - KS : ch;
-            const __nv_bfloat16* src = p.own[second ? 1 : 0] + grow_ * p.d + 16 * kk;
+            const __nv_bfloat16* src = p.own[C::XT0 + (second ? 1 : 0)] + grow_ * p.d + 16 * kk;
             v[i][0] = v[i][1] = make_uint4(0, 0, 0, 0);
             if (ch < 2 * KS && valid_ && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
             if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
@@ -242,7 +231,6 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             if (C::TRANSPOSED)
                 if (!ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after_sync();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 0);
             const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
             const int key0 = j * BC + 16 * sl;  // first stream row of this slice
             if (NPAIR == 1) {
@@ -326,15 +314,12 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     }
                 }
                 // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 2);
                 if (!ptx::mbar_wait(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 3);
                 uint32_t s3[16], s4[16];
                 ptx::tmem_ld16(sbase + 2 * BC, s3);
                 ptx::tmem_ld16(sbase + 3 * BC, s4);
                 ptx::tmem_wait_ld();
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 4);
                 uint32_t pa0[8], pa1[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
@@ -347,20 +332,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     pa0[k] = ptx::pack_bf16(w0, w1);
                     pa1[k] = ptx::pack_bf16(d0, d1);
                 }
-                if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 5);
                 ptx::tmem_st8(sbase + 2 * BC, pa0);
                 ptx::tmem_st8(sbase + 3 * BC, pa1);
             }
             ptx::tmem_wait_st();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 6);
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0 && q == 0 && sl == 0) BTL_STAMP(1, g, 1);
-            if (lane == 0) BTL_STAMP(4 + (w >> 3), g, w & 7);
             if (lane == 0) ptx::mbar_arrive(bar(C::B_PREADY + b));
         }
         if (!ok) break;
-        if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 0);  // tiles of the item done (warp 0)
         // the next item's operands, so that its loads and first score MMAs run under this item's epilogue
         if (item + (int)gridDim.x < items) {
             if (NPAIR == 1) {
@@ -371,9 +351,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             }
             stage_x(item + gridDim.x, it + 1);
         }
-        if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 2);  // next item's operands staged (warp 0)
         if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
-        if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 3);  // last output MMAs of the item done
         if (ok) {
             ptx::tc_fence_after_sync();
             __nv_bfloat16* p0 = p.out0 + grow * p.d;
@@ -398,7 +376,6 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     }
                 }
             }
-            if (lane == 0 && w == 0) BTL_STAMP(3, it + 1, 1);  // epilogue of the item done (warp 0)
         // the accumulators may be overwritten by the first output MMAs of the next item
             ptx::tc_fence_before_sync();
             __syncwarp();
@@ -417,7 +394,10 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     constexpr int BC = C::BC, KS = C::KS, NA = C::NA, SE = C::SE, SL = C::SL, NPAIR = C::NPAIR;
     // the next backward pass in the stream, if launched as a programmatic dependent, may start as SMs free up
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (*reinterpret_cast<volatile int*>(p.status) != 0) return;  // an earlier kernel timed out
+    if (*reinterpret_cast<volatile int*>(p.status) != 0) {  // an earlier kernel timed out
+        if (MODE != BWD_DV && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -489,7 +469,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 0) BTL_STAMP(3, 0, 0);
 
     // shared-memory address of tile j of streamed tensor t (0, 1: E ring; 2, 3: L ring)
     auto tile_addr = [&](int t, int j) -> uint32_t {
@@ -568,8 +547,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
                     }
                     if constexpr (NA == 2) {
-                        const __nv_bfloat16* o2 = p.own[2] + lane_row + (size_t)row0 * p.d;
-                        const __nv_bfloat16* o3 = p.own[3] + lane_row + (size_t)row0 * p.d;
+                        const __nv_bfloat16* o2 = p.own[C::XS0] + lane_row + (size_t)row0 * p.d;
+                        const __nv_bfloat16* o3 = p.own[C::XS0 + 1] + lane_row + (size_t)row0 * p.d;
                         const int rows_left = p.N - row0;
 #pragma unroll
                         for (int k = 0; k < KT; ++k) {
@@ -578,8 +557,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                 for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
                                     const bool v = lane + 32 * rp < rows_left;
                                     const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
-                                    ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[2], v ? 16u : 0u);
-                                    ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[3], v ? 16u : 0u);
+                                    ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[C::XS0], v ? 16u : 0u);
+                                    ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[C::XS0 + 1], v ? 16u : 0u);
                                 }
                             }
                         }
@@ -596,7 +575,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
-                            if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 3);
                             pend_s = -1;
                             if (ring == 0 && owner_pend) {  // cp.async groups complete in order: the owner copies have landed too
                                 if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
@@ -606,7 +584,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     }
                     ok = ptx::mbar_wait_warp(bar(b_empty + s), ph ^ 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     if (!ok) break;
-                    if (lane == 0 && ring == 0) BTL_STAMP(2, j, 0);
                     const uint32_t stage = ring_base + s * 2 * TB;
                     if (lane == 0) {
                         ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
@@ -646,13 +623,11 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                             }
                         }
                         ptx::cp_async_commit();
-                        if (lane == 0 && ring == 0) BTL_STAMP(2, j, 1);
                         if (pend_s >= 0) {  // the tile before: its copies have had a whole iteration to land
                             ptx::cp_async_wait<1>();
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
-                            if (lane == 0 && ring == 0) BTL_STAMP(2, j - 1, 2);
                             if (ring == 0 && owner_pend) {
                                 if (lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
                                 owner_pend = false;
@@ -716,7 +691,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // the first tiles of an item: its owner operands are in tensor memory
             if (j < 2 && !ptx::mbar_wait_warp(bar(C::B_QREADY + (it & 1)), (it >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
-            if (lane == 0) BTL_STAMP(0, g, 0);
             // Y0, Y1 in the E ring, K-major B
             const uint32_t t0 = tile_addr(0, g), t1 = tile_addr(1, g);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
@@ -731,12 +705,10 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 ptx::mma_ts_elect(dT, ax0 + 8 * kk, e_kdesc(t1, kk), idesc_s, 1u);
             ptx::mma_commit_elect(bar(C::B_SFULL + b));
             ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
-            if (lane == 0) BTL_STAMP(0, g, 1);
             return true;
         };
         auto issue_outputs = [&](int g, int it, int j) -> bool {  // DV only
             const int b = g & 1;
-            if (lane == 0) BTL_STAMP(0, g, 2);
             if (!ptx::mbar_wait_warp(bar(C::B_LFULL + g % SL), (g / SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             if (!ptx::mbar_wait_warp(bar(C::B_PREADY + b), (g >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             // the other issuer has queued its batch of tile g - 1: accumulation order is the tile order
@@ -744,7 +716,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             // the first tile of an item overwrites the accumulators: all sixteen element-wise warps have read them
             if (j == 0 && it > 0 && !ptx::mbar_wait_warp(bar(C::B_ACCFREE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
-            if (lane == 0) BTL_STAMP(0, g, 3);
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B (the L ring): atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
             const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);
@@ -760,7 +731,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
             ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
-            if (lane == 0) BTL_STAMP(0, g, 4);
             return true;
         };
         bool ok = true;
@@ -798,38 +768,40 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 //   (S, Sd)(0), (D, X)(0), then per tile j: (S, Sd)(j+1) once the element-wise warps have read
                 //   (S, Sd)(j) | outputs(j) once the operands W, dA are written | (D, X)(j+1), which overwrites them.
                 const uint32_t dS = tb + C::COL_SCORE, dT = dS + BC, dD = dS + 2 * BC, dX = dS + 3 * BC;
-                auto issue_first_pair = [&](int g) {  // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; Y0, Y1 in the L ring, K-major
+                // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; X0, X1 in shared memory, Y0, Y1 in the L ring, all K-major.
+                // `last`: the item's last tile; the shared-memory owner tiles are free once these MMAs are done
+                auto issue_first_pair = [&](int g, bool last) {
                     const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, g), 16, 1024);
                     const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, g), 16, 1024);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
                         const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ts_elect(dS, ax0 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                        ptx::mma_ss_elect(dS, own_kdesc(0, kk), y0 + off, idesc_s, kk > 0 ? 1u : 0u);
                     }
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
                         const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ts_elect(dT, ax1 + 8 * kk, y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                        ptx::mma_ss_elect(dT, own_kdesc(1, kk), y0 + off, idesc_s, kk > 0 ? 1u : 0u);
                     }
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
                         const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ts_elect(dT, ax0 + 8 * kk, y1 + off, idesc_s, 1u);
+                        ptx::mma_ss_elect(dT, own_kdesc(0, kk), y1 + off, idesc_s, 1u);
                     }
                     ptx::mma_commit_elect(bar(C::B_SFULL + 0));
+                    if (last) ptx::mma_commit_elect(bar(C::B_OWNFREE));
                 };
-                // `last`: the item's last tile; the shared-memory owner tiles are free once these MMAs are done
-                auto issue_second_pair = [&](int g, bool last) {  // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; Y2, Y3 in the E ring
+                // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; X2, X3 in tensor memory, Y2, Y3 in the E ring
+                auto issue_second_pair = [&](int g) {
                     const uint32_t t2 = tile_addr(0, g), t3 = tile_addr(1, g);
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dD, own_kdesc(0, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_elect(dD, ax0 + 8 * kk, e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(1, kk), e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_elect(dX, ax1 + 8 * kk, e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ss_elect(dX, own_kdesc(0, kk), e_kdesc(t3, kk), idesc_s, 1u);
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_elect(dX, ax0 + 8 * kk, e_kdesc(t3, kk), idesc_s, 1u);
                     ptx::mma_commit_elect(bar(C::B_SFULL + 1));
                     ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
-                    if (last) ptx::mma_commit_elect(bar(C::B_OWNFREE));
                 };
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int g0 = it * T;
@@ -842,8 +814,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     if (ok) ok = ptx::mbar_wait_warp(bar(C::B_EFULL + g0 % SE), (g0 / SE) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    issue_first_pair(g0);
-                    issue_second_pair(g0, T == 1);
+                    issue_first_pair(g0, T == 1);
+                    issue_second_pair(g0);
                     for (int j = 0; ok && j < T; ++j) {
                         const int g = g0 + j;
                         if (j + 1 < T) {
@@ -858,18 +830,14 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                 if (!ok) break;
                             }
                             ptx::tc_fence_after_sync();
-                            if (lane == 0) BTL_STAMP(0, gn, 0);
-                            issue_first_pair(gn);
-                            if (lane == 0) BTL_STAMP(0, gn, 1);
+                            issue_first_pair(gn, j + 2 == T);
                         }
                         // outputs(g): acc0 += W B0, acc1 += dA B0 + W B1 with the operands in the D and X columns
-                        if (lane == 0) BTL_STAMP(0, g, 2);
                         ok = ptx::mbar_wait_warp(bar(C::B_PREADY + 0), g & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                         // the first tile of an item overwrites the accumulators: the element-wise warps have read them
                         if (ok && j == 0 && it > 0) ok = ptx::mbar_wait_warp(bar(C::B_ACCFREE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
-                        if (lane == 0) BTL_STAMP(0, g, 3);
                         {
                             const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);  // MN-major B
                             const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
@@ -885,8 +853,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                             ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
                             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
                         }
-                        if (lane == 0) BTL_STAMP(0, g, 4);
-                        if (j + 1 < T) issue_second_pair(g + 1, j + 2 == T);
+                        if (j + 1 < T) issue_second_pair(g + 1);
                     }
                 }
             }
@@ -898,12 +865,15 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     // ---------------------------------------------------------------------- teardown
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0) BTL_STAMP(3, 0, 1);
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, 512);
     }
     if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, 1);
+    // DK and DQ start while the pass before them still runs (programmatic dependent launch) and read nothing it
+    // writes; they must still not complete before it, or completion of the last pass would not imply that the
+    // gradients of the earlier ones are written.  (No effect on a launch without the attribute.)
+    if (MODE != BWD_DV && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace tvm_attn

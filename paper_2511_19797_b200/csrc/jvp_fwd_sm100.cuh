@@ -66,7 +66,6 @@ struct FwdParams {
     float* lse;
     float* mu;
     int* status;  // device status word; non-zero makes the kernel a no-op
-    unsigned long long* tl;  // unused (timeline builds of other variants)
 };
 
 template <int DP>

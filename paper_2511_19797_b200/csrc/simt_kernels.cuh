@@ -157,28 +157,73 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
 
 // ------------------------------------------------------------------------------------------------
 // Backward pre-pass (App. C "Step 1", reduced by the identities Sigma_1 = rowsum(dtO*O),
-// Sigma_2 = rowsum(dtO*tO) and the standard-attention row term rowsum(dO*O)).  One warp per row.
-//   sig1[row] = sum_c Hc*O        cvec[row] = sum_c G*O + Hc*tO
+// Sigma_2 = rowsum(dtO*tO) and the standard-attention row term rowsum(dO*O)):
+//   sig1[row] = sum_c Hc*O        cvec[row] = sum_c G*O + Hc*tO        lse2[row] = lse[row] * log2(e)
+// Pure streaming work (four tensors read once), so it is laid out for the memory system: every lane
+// loads 16 bytes per tensor, a row is shared by the smallest power-of-two group of lanes that covers
+// its d * sizeof(T) / 16 chunks, and a warp has the loads of ROWSUM_UNROLL row groups in flight
+// before it touches the first.
+constexpr int ROWSUM_THREADS = 256;
+constexpr int ROWSUM_UNROLL = 2;
+
+__device__ __forceinline__ void dot_chunk(const uint4& a, const uint4& b, float& acc, float) {
+    const float* x = reinterpret_cast<const float*>(&a);
+    const float* y = reinterpret_cast<const float*>(&b);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc = fmaf(x[i], y[i], acc);
+}
+__device__ __forceinline__ void dot_chunk(const uint4& a, const uint4& b, float& acc, __nv_bfloat16) {
+    const __nv_bfloat162* x = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* y = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 xf = __bfloat1622float2(x[i]), yf = __bfloat1622float2(y[i]);
+        acc = fmaf(xf.x, yf.x, acc);
+        acc = fmaf(xf.y, yf.y, acc);
+    }
+}
+
+// `gs` = lanes per row (power of two, >= chunks per row `cpr`); rows_per_warp = 32 / gs.
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(ROWSUM_THREADS)
 bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* __restrict__ O,
                    const T* __restrict__ tO, const float* __restrict__ lse, float* __restrict__ sig1,
-                   float* __restrict__ cvec, float* __restrict__ lse2, long long rows, int d) {
-    const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= rows) return;
+                   float* __restrict__ cvec, float* __restrict__ lse2, long long rows, int d, int cpr, int gs) {
+    constexpr int VEC = 16 / (int)sizeof(T);
     const int lane = threadIdx.x & 31;
-    const size_t base = (size_t)row * d;
-    float s1 = 0.f, cc = 0.f;
-    for (int c = lane; c < d; c += 32) {
-        const float g = to_f32(G[base + c]), h = to_f32(Hc[base + c]);
-        const float o = to_f32(O[base + c]), to = to_f32(tO[base + c]);
-        s1 = fmaf(h, o, s1);
-        cc = fmaf(g, o, cc);
-        cc = fmaf(h, to, cc);
+    const int rpw = 32 / gs;                  // rows per warp and step
+    const int sub = lane / gs, c = lane - sub * gs;
+    const long long warp_id = (long long)blockIdx.x * (ROWSUM_THREADS / 32) + (threadIdx.x >> 5);
+    const long long row0 = warp_id * (ROWSUM_UNROLL * rpw) + sub;
+    uint4 g[ROWSUM_UNROLL], h[ROWSUM_UNROLL], o[ROWSUM_UNROLL], t[ROWSUM_UNROLL];
+    bool act[ROWSUM_UNROLL];
+#pragma unroll
+    for (int u = 0; u < ROWSUM_UNROLL; ++u) {
+        const long long row = row0 + (long long)u * rpw;
+        act[u] = row < rows && c < cpr;
+        if (act[u]) {
+            const size_t off = (size_t)row * d + (size_t)c * VEC;
+            g[u] = __ldg(reinterpret_cast<const uint4*>(G + off));
+            h[u] = __ldg(reinterpret_cast<const uint4*>(Hc + off));
+            o[u] = __ldg(reinterpret_cast<const uint4*>(O + off));
+            t[u] = __ldg(reinterpret_cast<const uint4*>(tO + off));
+        }
     }
-    s1 = warp_sum(s1);
-    cc = warp_sum(cc);
-    if (lane == 0) { sig1[row] = s1; cvec[row] = cc; lse2[row] = lse[row] * 1.4426950408889634f; }
+#pragma unroll
+    for (int u = 0; u < ROWSUM_UNROLL; ++u) {
+        const long long row = row0 + (long long)u * rpw;
+        float s1 = 0.f, cc = 0.f;
+        if (act[u]) {
+            dot_chunk(h[u], o[u], s1, T());
+            dot_chunk(g[u], o[u], cc, T());
+            dot_chunk(h[u], t[u], cc, T());
+        }
+        for (int off = gs >> 1; off > 0; off >>= 1) {
+            s1 += __shfl_xor_sync(0xffffffffu, s1, off);
+            cc += __shfl_xor_sync(0xffffffffu, cc, off);
+        }
+        if (c == 0 && row < rows) { sig1[row] = s1; cvec[row] = cc; lse2[row] = lse[row] * 1.4426950408889634f; }
+    }
 }
 
 // The four per-pair quantities of the backward from the six dot products of a (query, key) pair.

@@ -68,6 +68,10 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 // ---------------------------------------------------------------- TMA (tiled, 3-D, no multicast)
 __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
@@ -294,6 +298,26 @@ __device__ __forceinline__ bool mbar_test_warp(uint32_t bar, uint32_t parity) {
         : "r"(bar), "r"(parity)
         : "memory");
     return __all_sync(0xffffffffu, ok != 0);
+}
+
+// Bounded wait for two mbarrier phases, executed by a whole warp; warp-uniform result.  Both are polled back
+// to back first, so that when both have completed (the steady state of a pipeline) one shared-memory round
+// trip replaces two serial ones.
+__device__ __forceinline__ bool mbar_wait2_warp(uint32_t b0, uint32_t p0, uint32_t b1, uint32_t p1, volatile int* abort_flag,
+                                                uint64_t limit_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred a;\n\t.reg .pred b;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 a, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 b, [%3], %4;\n\t"
+        "and.pred a, a, b;\n\t"
+        "selp.u32 %0, 1, 0, a;\n\t}"
+        : "=r"(ok)
+        : "r"(b0), "r"(p0), "r"(b1), "r"(p1)
+        : "memory");
+    if (__all_sync(0xffffffffu, ok != 0)) return true;
+    if (!mbar_wait_warp(b0, p0, abort_flag, limit_ns)) return false;
+    return mbar_wait_warp(b1, p1, abort_flag, limit_ns);
 }
 
 // Non-blocking test of three mbarrier phases at once; the three polls are issued back to back so

@@ -19,24 +19,23 @@
 namespace tvm_attn {
 
 static std::atomic<uint64_t> g_launches{0};
-#ifdef TVM_ATTN_TIMELINE
-static unsigned long long* g_timeline = nullptr;  // clock stamps of CTA 0 (timeline builds only)
-#endif
 __device__ int g_status_word = 0;  // raised by a tensor-core kernel whose bounded wait ran out
 
-// Optional per-kernel timing: events recorded around each launch of the most recent call.
+// Optional per-kernel timing: events recorded around each launch of the most recent call.  While it is
+// disabled (the normal state) a call only reads the atomic flag, so concurrent calls from several host
+// threads do not touch shared state; while it is enabled the library is to be driven by one thread.
 struct Profiler {
-    bool enabled = false;
-    int count = 0;  // kernels recorded by the last call
+    std::atomic<bool> enabled{false};
+    std::atomic<int> count{0};  // kernels recorded by the last call
     cudaEvent_t ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-    void begin_call() { count = 0; }
+    void begin_call() { if (enabled.load(std::memory_order_relaxed)) count.store(0); }
     void mark(cudaStream_t st, int idx) {
-        if (!enabled || idx >= 8) return;
+        if (idx >= 8) return;
         if (!ev[idx] && cudaEventCreate(&ev[idx]) != cudaSuccess) { ev[idx] = nullptr; return; }
         cudaEventRecord(ev[idx], st);
     }
-    void before(cudaStream_t st) { if (enabled && count == 0) mark(st, 0); }
-    void after(cudaStream_t st) { if (enabled) { mark(st, count + 1); ++count; } }
+    void before(cudaStream_t st) { if (enabled.load(std::memory_order_relaxed) && count.load() == 0) mark(st, 0); }
+    void after(cudaStream_t st) { if (enabled.load(std::memory_order_relaxed)) { mark(st, count.load() + 1); count.fetch_add(1); } }
 };
 static Profiler g_prof;
 
@@ -93,10 +92,15 @@ template <typename T>
 static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const void* O, const void* tO, const float* lse,
                           float* sig1, float* cvec, float* lse2, cudaStream_t st) {
     const long long rows = s.BH * s.N;
-    const unsigned grid = (unsigned)((rows + 7) / 8);
+    const int cpr = s.d * (int)sizeof(T) / 16;  // 16-byte chunks per row (d % 8 == 0)
+    int gs = 1;
+    while (gs < cpr) gs <<= 1;
+    if (gs > 32) return TVM_ATTN_UNSUPPORTED;   // d <= 128 keeps a row within one warp
+    const long long rows_per_block = (long long)(ROWSUM_THREADS / 32) * ROWSUM_UNROLL * (32 / gs);
+    const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
     g_prof.before(st);
-    bwd_rowsums_kernel<T><<<grid, 256, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, lse, sig1, cvec,
-                                                lse2, rows, s.d);
+    bwd_rowsums_kernel<T><<<grid, ROWSUM_THREADS, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, lse, sig1,
+                                                           cvec, lse2, rows, s.d, cpr, gs);
     g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
@@ -239,7 +243,7 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
         prm.own[t] = static_cast<const __nv_bfloat16*>(own[t]);
     }
     for (int t = 0; t < 2; ++t) {
-        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? 2 + t : t], s, BWD_ROWS);
+        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? C::XS0 + t : t], s, BWD_ROWS);
         if (rc != TVM_ATTN_OK) return rc;
     }
     auto kern = jvp_bwd_kernel<MODE, DP>;
@@ -257,8 +261,10 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
         // DK and DQ read nothing that the pass before them writes (DV, DK and DQ all depend on the row-sums
         // pre-pass only, which has completed before DV starts), so their CTAs may fill the SMs that the last,
         // partial wave of the pass before leaves idle: programmatic dependent launch, with every CTA of these
-        // kernels releasing its dependents at once and none waiting for its primary.  Not while per-kernel
-        // events are being recorded: they would time overlapping kernels.
+        // kernels releasing its dependents at once.  None waits for its primary before it works; each waits for
+        // it once at the very end (griddepcontrol.wait in the teardown), so that DQ cannot complete before DK, nor
+        // DK before DV: work enqueued behind the call still sees all six gradients.  Not while per-kernel events
+        // are being recorded: they would time overlapping kernels.
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)grid);
         cfg.blockDim = dim3(BWD_THREADS);
@@ -268,7 +274,7 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = (MODE != BWD_DV && !g_prof.enabled) ? 1 : 0;
+        cfg.numAttrs = (MODE != BWD_DV && !g_prof.enabled.load(std::memory_order_relaxed)) ? 1 : 0;
         if (cudaLaunchKernelEx(&cfg, kern, ms[0], ms[1], ms[2], ms[3], mo[0], mo[1], prm) != cudaSuccess)
             return cuda_status(cudaGetLastError());
     }
@@ -289,10 +295,6 @@ static int launch_bwd_pass_dp(const Shape& s, const void* const own[4], const vo
     }
 }
 
-#ifdef TVM_ATTN_DEBUG_DUMP
-static float* g_debug_dump = nullptr;
-#endif
-
 static TcParams base_params(const Shape& s, int* status) {
     TcParams prm;
     std::memset(&prm, 0, sizeof prm);
@@ -301,9 +303,6 @@ static TcParams base_params(const Shape& s, int* status) {
     prm.c2 = s.alpha * 1.4426950408889634f;
     prm.out_scale = 1.0f;
     prm.status = status;
-#ifdef TVM_ATTN_DEBUG_DUMP
-    prm.dbg = g_debug_dump;
-#endif
     return prm;
 }
 
@@ -327,6 +326,24 @@ static int noalloc_scratch_address(float** out) {
     }
     *out = g_noalloc_addr[dev];
     return TVM_ATTN_OK;
+}
+
+// One warp waits, with a limit, on an mbarrier that nobody arrives at: the same bounded wait the tensor-core
+// kernels use, made to run out on purpose so that the time-out reporting can be exercised without disturbing
+// a real kernel.  Raises the device status word like they do.
+__global__ void selftest_timeout_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ __align__(8) unsigned long long barrier;
+    __shared__ int abort_flag;
+    if (*reinterpret_cast<volatile int*>(status) != 0) return;
+    const uint32_t bar = ptx::smem_u32(&barrier);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ptx::mbar_init(bar, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncwarp();
+    const bool ok = ptx::mbar_wait_warp(bar, 0, &abort_flag, limit_ns);
+    if (!ok && threadIdx.x == 0 && abort_flag) atomicExch(status, 1);
 }
 
 }  // namespace tvm_attn
@@ -370,11 +387,6 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
         f.Q = static_cast<const __nv_bfloat16*>(Q); f.tQ = static_cast<const __nv_bfloat16*>(tQ);
         f.K = static_cast<const __nv_bfloat16*>(K); f.tK = static_cast<const __nv_bfloat16*>(tK);
         f.V = static_cast<const __nv_bfloat16*>(V); f.tV = static_cast<const __nv_bfloat16*>(tV);
-#ifdef TVM_ATTN_TIMELINE
-        f.tl = g_timeline;
-#else
-        f.tl = nullptr;
-#endif
         f.O = static_cast<__nv_bfloat16*>(O); f.tO = static_cast<__nv_bfloat16*>(tO);
         f.lse = lse; f.mu = mu; f.status = status;
         switch (s.dp) {
@@ -430,9 +442,6 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         b.N = s.N; b.d = s.d; b.BH = (int)s.BH;
         b.alpha = s.alpha; b.c2 = s.alpha * 1.4426950408889634f;
         b.lse2 = lse2; b.mu = mu; b.sig1 = sig1; b.cvec = cvec; b.status = status;
-#ifdef TVM_ATTN_TIMELINE
-        b.tl = g_timeline;  // each pass gets its own third of the buffer (see below)
-#endif
         {   // dtV = P^T Hc, dV = P^T G + (P*Nn)^T Hc : owner keys (K, tK); stream queries (Q, tQ | Hc, G)
             BwdParams q = b; q.out_scale = 1.0f;
             q.out0 = static_cast<__nv_bfloat16*>(dtV); q.out1 = static_cast<__nv_bfloat16*>(dV);
@@ -443,7 +452,6 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         }
         {   // dtK = alpha W^T Q, dK = alpha (dA^T Q + W^T tQ) : owner keys (K, tK, V, tV); stream (Hc, G | Q, tQ)
             BwdParams q = b; q.out_scale = s.alpha;
-            if (q.tl) q.tl += 6 * 64 * 8;
             q.out0 = static_cast<__nv_bfloat16*>(dtK); q.out1 = static_cast<__nv_bfloat16*>(dK);
             const void* own[4] = {K, tK, V, tV};
             const void* strm[4] = {dtO, dO, Q, tQ};
@@ -452,7 +460,6 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         }
         {   // dtQ = alpha W K, dQ = alpha (dA K + W tK) : owner queries (Q, tQ, Hc, G); stream (V, tV | K, tK)
             BwdParams q = b; q.out_scale = s.alpha;
-            if (q.tl) q.tl += 2 * 6 * 64 * 8;
             q.out0 = static_cast<__nv_bfloat16*>(dtQ); q.out1 = static_cast<__nv_bfloat16*>(dQ);
             const void* own[4] = {Q, tQ, dtO, dO};
             const void* strm[4] = {V, tV, K, tK};
@@ -512,15 +519,25 @@ int tvm_attn_check_status(void* cuda_stream) {
     return TVM_ATTN_OK;
 }
 
+int tvm_attn_selftest_timeout(uint64_t limit_ns, void* cuda_stream) {
+    if (limit_ns == 0 || limit_ns > 100ull * 1000ull * 1000ull) return TVM_ATTN_INVALID_ARG;
+    int* status = status_word_ptr();
+    if (!status) return TVM_ATTN_CUDA_ERROR;
+    selftest_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(status, limit_ns);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
 int tvm_attn_set_profiling(int enable) {
-    g_prof.enabled = enable != 0;
-    g_prof.count = 0;
+    g_prof.enabled.store(enable != 0);
+    g_prof.count.store(0);
     return TVM_ATTN_OK;
 }
 
 int tvm_attn_get_profile(float* ms, int capacity) {
     if (!ms || capacity < 0) return TVM_ATTN_INVALID_ARG;
-    int n = g_prof.count < capacity ? g_prof.count : capacity;
+    const int recorded = g_prof.count.load();
+    int n = recorded < capacity ? recorded : capacity;
     if (n > 7) n = 7;
     if (n > 0 && cudaEventSynchronize(g_prof.ev[n]) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
     for (int k = 0; k < n; ++k)
@@ -545,12 +562,5 @@ const char* tvm_attn_strerror(int code) {
 }
 
 int tvm_attn_version(void) { return 100; }
-
-#ifdef TVM_ATTN_DEBUG_DUMP
-void tvm_attn_debug_set_dump(float* device_ptr) { g_debug_dump = device_ptr; }
-#endif
-#ifdef TVM_ATTN_TIMELINE
-void tvm_attn_debug_set_timeline(unsigned long long* device_ptr) { g_timeline = device_ptr; }
-#endif
 
 }  // extern "C"

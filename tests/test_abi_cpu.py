@@ -28,15 +28,31 @@ def test_header_functions_are_all_exported(lib):
     assert {"tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_jvp_workspace_bytes"} <= set(names)
     for n in names:
         assert hasattr(lib, n), "library does not export %s" % n
-    assert set(names) == set(binding.EXPORTS) | (set(names) - set(binding.EXPORTS))
-    for n in binding.EXPORTS:
-        assert n in names
+    assert set(names) == set(binding.EXPORTS), "the binding's export list and the header disagree"
 
 
 def test_version_and_strerror(lib):
     assert lib.tvm_attn_version() >= 100
-    for code in (0, -1, -2, -3, -4, -5, -99):
-        assert len(lib.tvm_attn_strerror(code)) > 0
+    texts = [lib.tvm_attn_strerror(code) for code in (0, -1, -2, -3, -4, -5, -6)]
+    assert all(len(t) > 0 for t in texts) and len(set(texts)) == len(texts)
+    assert lib.tvm_attn_strerror(-99) == lib.tvm_attn_strerror(-1234)     # unknown codes share one text
+    assert b"NOALLOC" in lib.tvm_attn_strerror(-6)
+
+
+def test_noalloc_backward_rejects_problems_beyond_its_scratch_before_any_gpu_work(lib):
+    rows = binding.NOALLOC_MAX_ROWS
+    ptrs = [ctypes.c_void_p(4096 + 16 * k) for k in range(18)]     # never dereferenced: the size check comes first
+    over = binding.Params(1, 1, rows + 8, 64, 0.0, binding.BF16, 0)
+    assert lib.tvm_attn_jvp_bwd_noalloc(ctypes.byref(over), *ptrs, None) == -6
+    over = binding.Params(16, 16, 1025, 72, 0.0, binding.BF16, 0)
+    assert lib.tvm_attn_jvp_bwd_noalloc(ctypes.byref(over), *ptrs, None) == -6
+    bad = binding.Params(1, 1, 64, 36, 0.0, binding.BF16, 0)
+    assert lib.tvm_attn_jvp_bwd_noalloc(ctypes.byref(bad), *ptrs, None) == -2   # shape errors come first
+
+
+def test_selftest_timeout_rejects_limits_out_of_range(lib):
+    assert lib.tvm_attn_selftest_timeout(0, None) == -1
+    assert lib.tvm_attn_selftest_timeout(10**9, None) == -1
 
 
 def test_workspace_bytes_host_only():

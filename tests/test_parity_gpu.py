@@ -4,8 +4,11 @@ same seeded inputs.  Error metric per tensor: max|gpu - ref| / max|ref|.
 Tolerances: bf16 mode 1e-2 for O and tO, 2e-2 for the six gradients (inputs are rounded to bf16
 once and the oracle consumes those rounded values, so only the kernels' own rounding counts);
 fp32 validation mode 1e-4 for everything.  The saved statistics lse and mu are fp32 in both modes;
-in bf16 mode they are held to 2e-3 (they come from bf16 tensor-core products accumulated in fp32).
+in bf16 mode they are held to 1e-4 as well: they are fp32 sums of exact products of the bf16 inputs, and only
+mu passes through one more rounding (the exponentials that weight it).
 """
+import threading
+
 import numpy as np
 import pytest
 import torch
@@ -15,7 +18,7 @@ from tests._parity import assert_within, run_case
 
 pytestmark = pytest.mark.gpu
 
-BF16_FWD, BF16_BWD, BF16_STATS, FP32_TOL = 1e-2, 2e-2, 2e-3, 1e-4
+BF16_FWD, BF16_BWD, BF16_STATS, FP32_TOL = 1e-2, 2e-2, 1e-4, 1e-4
 
 
 def test_tiny_fp32_validation_mode():
@@ -131,12 +134,17 @@ def test_errors_reported_on_the_gpu_box():
     assert binding.tvm_attn_launch_count() >= 0
 
 
+def test_longest_sequence_whole_heads():
+    """The longest sweep point as it is benchmarked (B=4, H=16, N=16384, d=64: 8192 work items of 256 stream
+    tiles each, dozens per CTA), all ten outputs element by element on four whole heads.  The C oracle takes a
+    few minutes per head on one core; the four heads run on four threads."""
+    errs, _, _ = run_case("sweep16384", oracle_heads=[0, 21, 42, 63])
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
 def test_longest_sequence_on_sampled_query_rows():
-    """N = 16384 (the longest sweep point) on a reduced batch: whole heads are too slow for the CPU oracle, but
-    the numpy oracle accepts fewer query rows than keys, so sampled rows of O, tO, lse, mu, dQ and dtQ are
-    compared element by element; the key-side gradients are checked through the identity
-    sum_j dV_j = sum_i (G_i + Hc_i (sum_j Pd_ij)) = sum_i G_i  (rows of P sum to 1, rows of Pd to 0)
-    and sum_j dtV_j = sum_i Hc_i, which hold at any size."""
+    """N = 16384 on a reduced batch, query-side outputs on sampled rows against the whole-matrix numpy oracle
+    (which accepts fewer query rows than keys): a second, independent writing of the definitions at this length."""
     from oracle import attn_jvp_numpy as onp
     wl = inputs.custom(1, 2, 16384, 64, seed=4, tangent_std=0.5)
     x = {k: v.to(torch.bfloat16) for k, v in inputs.make_inputs(wl).items()}
@@ -157,8 +165,87 @@ def test_longest_sequence_on_sampled_query_rows():
     errs = {"O": rel_err(pick(O), rO), "tO": rel_err(pick(tO), rtO), "lse": rel_err(pick(lse), rlse),
             "mu": rel_err(pick(mu), rmu), "dQ": rel_err(pick(grads[0]), rdQ), "dtQ": rel_err(pick(grads[3]), rdtQ)}
     assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
-    dV, dtV = grads[2].double().sum(dim=2).cpu(), grads[5].double().sum(dim=2).cpu()
-    sG, sH = x["dO"].double().sum(dim=2), x["dtO"].double().sum(dim=2)
-    scale = float(sG.abs().max())
-    assert float((dV - sG).abs().max()) <= BF16_BWD * max(scale, 1.0) * 8  # sums of N bf16-rounded rows
-    assert float((dtV - sH).abs().max()) <= BF16_BWD * max(float(sH.abs().max()), 1.0) * 8
+
+
+def test_gradients_are_complete_for_work_enqueued_behind_the_call():
+    """The three tensor-core passes of one backward call overlap (the later ones start while the earlier ones
+    drain).  Work enqueued on the same stream right after the call, with no host synchronisation in between,
+    must still see all six gradients complete."""
+    wl = inputs.custom(4, 37, 320, 72, seed=77)          # one wave is not enough: the passes do overlap
+    x = {k: v.to(torch.bfloat16).cuda() for k, v in inputs.make_inputs(wl).items()}
+    O, tO, lse, mu = binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"])
+    args = (x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], O, tO, lse, mu, x["dO"], x["dtO"])
+    for _ in range(3):
+        out = tuple(torch.full_like(x["Q"], float("nan")) for _ in range(6))
+        torch.cuda.synchronize()
+        binding.tvm_attn_jvp_bwd(*args, out=out)
+        seen = [t.clone() for t in out]                   # consumer kernels on the same stream, no sync before them
+        torch.cuda.synchronize()
+        binding.tvm_attn_check_status()
+        for name, a, b in zip(("dQ", "dK", "dV", "dtQ", "dtK", "dtV"), seen, out):
+            assert torch.isfinite(a.float()).all(), name
+            assert torch.equal(a, b), name
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_later_kernels_are_no_ops():
+    """Failure reporting, exercised without disturbing a real kernel: a one-warp kernel waits (1 ms limit) on a
+    barrier nobody signals, gives up and raises the device status.  A forward enqueued behind it must not touch
+    its outputs; the status is reported once and cleared; the next forward works."""
+    wl = inputs.custom(1, 2, 200, 72, seed=12)
+    x = {k: v.to(torch.bfloat16).cuda() for k, v in inputs.make_inputs(wl).items()}
+    ref = binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"])
+    assert binding.tvm_attn_check_status(raise_on_error=False) == 0
+    O, tO = torch.full_like(x["Q"], 7.0), torch.full_like(x["Q"], 7.0)
+    lse = torch.full(x["Q"].shape[:3], 7.0, device="cuda")
+    mu = torch.full_like(lse, 7.0)
+    binding.tvm_attn_selftest_timeout(1_000_000)
+    binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], out=(O, tO, lse, mu))
+    assert binding.tvm_attn_check_status(raise_on_error=False) == -5          # DEVICE_TIMEOUT
+    for t in (O, tO, lse, mu):
+        assert torch.all(t == 7.0), "a kernel behind the time-out wrote its outputs"
+    assert binding.tvm_attn_check_status(raise_on_error=False) == 0           # reported once, then cleared
+    with pytest.raises(binding.TvmAttnError):
+        binding.tvm_attn_selftest_timeout(0)
+    got = binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], out=(O, tO, lse, mu))
+    binding.tvm_attn_check_status()
+    for a, b in zip(got, ref):
+        assert torch.equal(a, b)
+
+
+def test_two_host_threads_on_two_streams():
+    """Concurrent calls from two host threads, each on its own stream with its own buffers and workspace, give
+    the results of the same calls made one after the other."""
+    wls = [inputs.custom(2, 9, 260, 72, seed=41), inputs.custom(3, 5, 200, 64, seed=42)]
+    xs = [{k: v.to(torch.bfloat16).cuda() for k, v in inputs.make_inputs(wl).items()} for wl in wls]
+
+    def run(x, stream):
+        with torch.cuda.stream(stream):
+            fw = binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], stream=stream)
+            gr = binding.tvm_attn_jvp_bwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], *fw, x["dO"], x["dtO"],
+                                          stream=stream)
+        return tuple(fw) + tuple(gr)
+
+    serial = [run(x, torch.cuda.current_stream()) for x in xs]
+    torch.cuda.synchronize()
+    results, errors = [None, None], []
+
+    def worker(i):
+        try:
+            st = torch.cuda.Stream()
+            for _ in range(5):
+                results[i] = run(xs[i], st)
+            st.synchronize()
+        except Exception as e:  # noqa: BLE001
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    binding.tvm_attn_check_status()
+    for i in range(2):
+        for a, b in zip(results[i], serial[i]):
+            assert torch.equal(a, b)
