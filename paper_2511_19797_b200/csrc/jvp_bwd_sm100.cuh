@@ -224,12 +224,15 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         for (int j = NPAIR == 1 ? ((par ^ g0) & 1) : 0; j < T; j += jstep) {
             const int g = g0 + j;
             const int b = NPAIR == 1 ? (g & 1) : 0, sph = NPAIR == 1 ? (g >> 1) & 1 : (g & 1);
-            if (!ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             // the statistics of the tile's queries arrive with its L stage, which is not released before the
-            // output MMAs of this tile, hence not before every warp is through with them
+            // output MMAs of this tile, hence not before every warp is through with them.  Every wait of these
+            // warps is warp-uniform: the tensor-memory accesses behind it need the whole warp.
             const float* st = stats + (g % C::SL) * 4 * 64 + 16 * sl;
-            if (C::TRANSPOSED)
-                if (!ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            if (C::TRANSPOSED) {
+                if (!ptx::mbar_wait2_warp(bar(C::B_SFULL + b), sph, bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            } else {
+                if (!ptx::mbar_wait_warp(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+            }
             ptx::tc_fence_after_sync();
             const uint32_t sbase = lane_addr + C::COL_SCORE + b * C::SCORE_BUF_COLS + 16 * sl;
             const int key0 = j * BC + 16 * sl;  // first stream row of this slice
@@ -314,7 +317,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     }
                 }
                 // ---- phase B: W = P D - P Sigma1, dA = (P X - P c) + W Nn, written over this slice's D and X columns
-                if (!ptx::mbar_wait(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                if (!ptx::mbar_wait_warp(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
                 uint32_t s3[16], s4[16];
                 ptx::tmem_ld16(sbase + 2 * BC, s3);
@@ -347,11 +350,11 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 // DV: this warp has seen only the scores of its own tiles; those of the item's last tile, which
                 // may belong to the other eight warps, must be complete too before the operands change
                 const int gl = g0 + T - 1;
-                if (!ptx::mbar_wait(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
+                if (!ptx::mbar_wait_warp(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             }
             stage_x(item + gridDim.x, it + 1);
         }
-        if (ok) ok = ptx::mbar_wait(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+        if (ok) ok = ptx::mbar_wait_warp(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
         if (ok) {
             ptx::tc_fence_after_sync();
             __nv_bfloat16* p0 = p.out0 + grow * p.d;
@@ -676,11 +679,6 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             return kk < 4 ? ptx::smem_desc_sw128(tile, 16, 1024) + (uint64_t)((kk * 32) >> 4)
                           : ptx::smem_desc_nosw(tile + BC * 128, BC * 16, 128);
         };
-        auto own_kdesc = [&](int t, int kk) -> uint64_t {
-            const uint32_t base = own_base + t * C::OWN_BYTES;
-            return kk < 4 ? ptx::smem_desc_sw128(base, 16, 1024) + (uint64_t)((kk * 32) >> 4)
-                          : ptx::smem_desc_nosw(base + BWD_ROWS * 128, BWD_ROWS * 16, 128);
-        };
         // tiles this CTA streams over all of its items; tile g belongs to item g / T of this CTA
         const int n_it = (int)blockIdx.x < items ? (items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
         const int G = n_it * T;
@@ -768,40 +766,60 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 //   (S, Sd)(0), (D, X)(0), then per tile j: (S, Sd)(j+1) once the element-wise warps have read
                 //   (S, Sd)(j) | outputs(j) once the operands W, dA are written | (D, X)(j+1), which overwrites them.
                 const uint32_t dS = tb + C::COL_SCORE, dT = dS + BC, dD = dS + 2 * BC, dX = dS + 3 * BC;
+                // One election per batch of MMAs and descriptors as 32-bit halves (see mma_ts_p): the issuing warp
+                // shares its scheduler with four element-wise warps, and every instruction it saves per MMA shortens
+                // the chain second pair -> phase B -> outputs -> second pair.  (DV and the forward, whose chains
+                // are not bound by the issue, measured 2 to 4 % slower this way and keep the elected-lane form.)
+                constexpr uint32_t HI_SW = ptx::desc_hi_sw128(1024), HI_E4 = ptx::desc_hi_nosw(128);
+                // k-step kk of a K-major tile whose columns from 64 on sit in an unswizzled block behind the atom
+                auto klo = [&](uint32_t tile, int rows, int kk) -> uint32_t {
+                    return kk < 4 ? ptx::desc_lo(tile, 16) + 2u * kk : ptx::desc_lo(tile + rows * 128, rows * 16);
+                };
                 // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; X0, X1 in shared memory, Y0, Y1 in the L ring, all K-major.
                 // `last`: the item's last tile; the shared-memory owner tiles are free once these MMAs are done
                 auto issue_first_pair = [&](int g, bool last) {
-                    const uint64_t y0 = ptx::smem_desc_sw128(tile_addr(2, g), 16, 1024);
-                    const uint64_t y1 = ptx::smem_desc_sw128(tile_addr(3, g), 16, 1024);
+                    const uint32_t el = ptx::elect_one();
+                    const uint32_t y0 = ptx::desc_lo(tile_addr(2, g), 16), y1 = ptx::desc_lo(tile_addr(3, g), 16);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
-                        const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ss_elect(dS, own_kdesc(0, kk), y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                        const uint32_t off = (uint32_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                        const uint32_t ahi = kk < 4 ? HI_SW : HI_E4;
+                        if (kk == 0) ptx::mma_ss_p<0>(el, dS, klo(own_base, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
+                        else ptx::mma_ss_p<1>(el, dS, klo(own_base, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
                     }
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
-                        const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ss_elect(dT, own_kdesc(1, kk), y0 + off, idesc_s, kk > 0 ? 1u : 0u);
+                        const uint32_t off = (uint32_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                        const uint32_t ahi = kk < 4 ? HI_SW : HI_E4;
+                        if (kk == 0) ptx::mma_ss_p<0>(el, dT, klo(own_base + C::OWN_BYTES, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
+                        else ptx::mma_ss_p<1>(el, dT, klo(own_base + C::OWN_BYTES, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
                     }
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
-                        const uint64_t off = (uint64_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ss_elect(dT, own_kdesc(0, kk), y1 + off, idesc_s, 1u);
+                        const uint32_t off = (uint32_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
+                        ptx::mma_ss_p<1>(el, dT, klo(own_base, BWD_ROWS, kk), kk < 4 ? HI_SW : HI_E4, y1 + off, HI_SW, idesc_s);
                     }
-                    ptx::mma_commit_elect(bar(C::B_SFULL + 0));
-                    if (last) ptx::mma_commit_elect(bar(C::B_OWNFREE));
+                    ptx::mma_commit_p(el, bar(C::B_SFULL + 0));
+                    if (last) ptx::mma_commit_p(el, bar(C::B_OWNFREE));
                 };
                 // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; X2, X3 in tensor memory, Y2, Y3 in the E ring
                 auto issue_second_pair = [&](int g) {
+                    const uint32_t el = ptx::elect_one();
                     const uint32_t t2 = tile_addr(0, g), t3 = tile_addr(1, g);
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_elect(dD, ax0 + 8 * kk, e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+                    for (int kk = 0; kk < KS; ++kk) {
+                        if (kk == 0) ptx::mma_ts_p<0>(el, dD, ax0 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                        else ptx::mma_ts_p<1>(el, dD, ax0 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                    }
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_elect(dX, ax1 + 8 * kk, e_kdesc(t2, kk), idesc_s, kk > 0 ? 1u : 0u);
+                    for (int kk = 0; kk < KS; ++kk) {
+                        if (kk == 0) ptx::mma_ts_p<0>(el, dX, ax1 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                        else ptx::mma_ts_p<1>(el, dX, ax1 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                    }
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_elect(dX, ax0 + 8 * kk, e_kdesc(t3, kk), idesc_s, 1u);
-                    ptx::mma_commit_elect(bar(C::B_SFULL + 1));
-                    ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_p<1>(el, dX, ax0 + 8 * kk, klo(t3, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                    ptx::mma_commit_p(el, bar(C::B_SFULL + 1));
+                    ptx::mma_commit_p(el, bar(C::B_EEMPTY + g % SE));
                 };
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int g0 = it * T;
@@ -839,19 +857,23 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
                         {
-                            const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);  // MN-major B
-                            const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
+                            const uint32_t el = ptx::elect_one();
+                            const uint32_t b0 = ptx::desc_lo(tile_addr(2, g), BC * 128), b1 = ptx::desc_lo(tile_addr(3, g), BC * 128);  // MN-major B
                             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
 #pragma unroll
                             for (int u = 0; u < BC / 16; ++u) {
-                                const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
-                                const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                                ptx::mma_ts_elect(acc0, dD + 16 * u, b0 + off, idesc_o, acc);
-                                ptx::mma_ts_elect(acc1, dX + 16 * u, b0 + off, idesc_o, acc);
-                                ptx::mma_ts_elect(acc1, dD + 16 * u, b1 + off, idesc_o, 1u);
+                                const uint32_t off = (uint32_t)((u * 16 * 128) >> 4);
+                                if (u == 0 && j == 0) {
+                                    ptx::mma_ts_p<0>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                } else {
+                                    ptx::mma_ts_p<1>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                }
+                                ptx::mma_ts_p<1>(el, acc1, dD + 16 * u, b1 + off, HI_SW, idesc_o);
                             }
-                            ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
-                            if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
+                            ptx::mma_commit_p(el, bar(C::B_LEMPTY + g % SL));
+                            if (j == T - 1) ptx::mma_commit_p(el, bar(C::B_FINAL));
                         }
                         if (j + 1 < T) issue_second_pair(g + 1);
                     }

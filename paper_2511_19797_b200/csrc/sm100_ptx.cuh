@@ -251,6 +251,51 @@ __device__ __forceinline__ void mma_commit_elect(uint32_t bar) {
         "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
         ::"r"(bar) : "memory");
 }
+// Batched issue: one election per batch of MMAs instead of one per MMA, and descriptors handled as two 32-bit
+// halves.  Only the low half (start address and leading offset) changes from MMA to MMA, so stepping through
+// k-steps or tiles is one 32-bit add; the high half holds the stride offset, the descriptor version and the
+// swizzle mode.  `el` is non-zero on the one elected lane.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\tselp.u32 %0, 1, 0, e;\n\t}" : "=r"(r));
+    return r;
+}
+__host__ __device__ constexpr uint32_t desc_hi_sw128(uint32_t sbo_bytes) { return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29); }
+__host__ __device__ constexpr uint32_t desc_hi_nosw(uint32_t sbo_bytes) { return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14); }
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+template <uint32_t ACC>
+__device__ __forceinline__ void mma_ts_p(uint32_t el, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .pred e;\n\t.reg .b64 b;\n\t"
+        "setp.ne.b32 e, %0, 0;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 b, {%3, %4};\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], b, %5, p;\n\t}"
+        ::"r"(el), "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC)
+        : "memory");
+}
+template <uint32_t ACC>
+__device__ __forceinline__ void mma_ss_p(uint32_t el, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .pred e;\n\t.reg .b64 a;\n\t.reg .b64 b;\n\t"
+        "setp.ne.b32 e, %0, 0;\n\t"
+        "setp.ne.b32 p, %7, 0;\n\t"
+        "mov.b64 a, {%2, %3};\n\t"
+        "mov.b64 b, {%4, %5};\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %6, p;\n\t}"
+        ::"r"(el), "r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit_p(uint32_t el, uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .pred e;\n\t"
+        "setp.ne.b32 e, %0, 0;\n\t"
+        "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
+        ::"r"(el), "r"(bar) : "memory");
+}
+
 // Bounded wait executed by a whole warp; the result is made warp-uniform.  (All lanes poll: letting
 // lane 0 poll alone and broadcasting its verdict measured slower.)
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
