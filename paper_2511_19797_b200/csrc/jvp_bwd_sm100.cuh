@@ -228,7 +228,13 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             // output MMAs of this tile, hence not before every warp is through with them.  Every wait of these
             // warps is warp-uniform: the tensor-memory accesses behind it need the whole warp.
             const float* st = stats + (g % C::SL) * 4 * 64 + 16 * sl;
-            if (C::TRANSPOSED) {
+            if (NPAIR == 1) {
+                // DV waits here for scores that are usually not there yet: a blocking wait, then the statistics'
+                // barrier (long complete), and one vote for both
+                bool okl = ptx::mbar_wait(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS);
+                if (okl) okl = ptx::mbar_wait(bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS);
+                if (!__all_sync(0xffffffffu, okl)) { ok = false; break; }
+            } else if (C::TRANSPOSED) {
                 if (!ptx::mbar_wait2_warp(bar(C::B_SFULL + b), sph, bar(C::B_LFULL + g % C::SL), (g / C::SL) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             } else {
                 if (!ptx::mbar_wait_warp(bar(C::B_SFULL + b), sph, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
@@ -453,12 +459,13 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
             for (int i = threadIdx.x; i < SE * 2 * BC; i += BWD_THREADS) {  // E ring: second chunk block
                 const int t = i / BC, r = i - t * BC;
-                *reinterpret_cast<uint4*>(smem + C::NOWN_SMEM * C::OWN_BYTES + t * C::EST_BYTES + BC * 128 + BC * 16 + r * 16) =
-                    make_uint4(0, 0, 0, 0);
+                // stage t / 2, tensor t & 1: second chunk block of the stage's tail area
+                *reinterpret_cast<uint4*>(smem + C::NOWN_SMEM * C::OWN_BYTES + (t >> 1) * 2 * C::EST_BYTES + 2 * BC * 128 + 2 * BC * 16 +
+                                          (t & 1) * BC * 16 + r * 16) = make_uint4(0, 0, 0, 0);
             }
             for (int i = threadIdx.x; i < SL * 2 * BC; i += BWD_THREADS) {  // L ring: chunk 1 of the second swizzle atom
                 const int t = i / BC, r = i - t * BC;
-                uint8_t* atom2 = smem + C::NOWN_SMEM * C::OWN_BYTES + SE * 2 * C::EST_BYTES + t * C::LST_BYTES + BC * 128;
+                uint8_t* atom2 = smem + C::NOWN_SMEM * C::OWN_BYTES + SE * 2 * C::EST_BYTES + (t >> 1) * 2 * C::LST_BYTES + (2 + (t & 1)) * BC * 128;
                 *reinterpret_cast<uint4*>(atom2 + r * 128 + ((1 ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
             }
             ptx::fence_proxy_async_smem();
@@ -473,10 +480,12 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    // shared-memory address of tile j of streamed tensor t (0, 1: E ring; 2, 3: L ring)
-    auto tile_addr = [&](int t, int j) -> uint32_t {
-        return t < 2 ? e_base + ((j % SE) * 2 + t) * C::EST_BYTES : l_base + ((j % SL) * 2 + (t - 2)) * C::LST_BYTES;
-    };
+    // Shared-memory stage of tile j in the E and the L ring.  A stage holds the tile's two tensors interleaved so
+    // that, read K-major, the two form ONE operand of 2 * BC rows (a score MMA with N = 128 then covers both):
+    //   E stage: [Y0 atom][Y1 atom][tail chunk 0: Y0 rows, Y1 rows][tail chunk 1: Y0 rows, Y1 rows]   (tail: NA == 2)
+    //   L stage: [Y0 atom 0][Y1 atom 0][Y0 atom 1][Y1 atom 1]                                            (atom 1: NA == 2)
+    auto e_stage = [&](int j) -> uint32_t { return e_base + (j % SE) * 2 * C::EST_BYTES; };
+    auto l_stage = [&](int j) -> uint32_t { return l_base + (j % SL) * 2 * C::LST_BYTES; };
 
     if (warp == 0 || warp == 2) {
         // ------------------------------------------------------------------ producers: warp 0 feeds the E
@@ -506,7 +515,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
             // Destination of chunk 0 of row `lane` behind the 64-column atom: the E ring keeps compact
             // 16-byte-per-row blocks (K-major operands only), the L ring a second 128-byte-swizzled atom.
-            [[maybe_unused]] const uint32_t dst_lane = BC * 128 + (ring == 0 ? lane * 16 : lane * 128);
+            [[maybe_unused]] const uint32_t dst_lane = 2 * BC * 128 + (ring == 0 ? lane * 16 : lane * 128);
             [[maybe_unused]] const uint32_t sw = lane & 7;  // rows 32 apart share it
             // statistics: 16-byte chunks when the rows of the (B, H, N) arrays are 16-byte aligned, else floats
             const bool st16 = (p.N & 3) == 0;
@@ -591,7 +600,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     if (lane == 0) {
                         ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
                         ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
-                        ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
+                        ptx::tma_load_3d(stage + BC * 128, map1, bar(b_full + s), 0, j * BC, bh);
                     }
                     if constexpr (HAS_CP) {
                         [[maybe_unused]] const int rows_left = p.N - j * BC;  // rows of this tile that exist
@@ -619,9 +628,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                 for (int rp = 0; rp < BC / 32; ++rp) {
                                     const bool v = lane + 32 * rp < rows_left;
                                     const uint32_t dst = stage + dst_lane +
-                                                         (ring == 0 ? k * BC * 16 + rp * 32 * 16 : rp * 32 * 128 + ((k ^ sw) << 4));
+                                                         (ring == 0 ? k * 2 * BC * 16 + rp * 32 * 16 : rp * 32 * 128 + ((k ^ sw) << 4));
                                     ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
-                                    ptx::cp_async_16(dst + TB, v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                                    ptx::cp_async_16(dst + (ring == 0 ? BC * 16 : BC * 128), v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
                                 }
                             }
                         }
@@ -672,13 +681,29 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         constexpr uint32_t idesc_o = ptx::idesc_bf16_f32(128, DP, 0, 1);
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);  // warp-uniform for the compiler
         const uint32_t ax0 = tb + C::COL_X0, ax1 = tb + C::COL_X1;
-        // owner tiles in shared memory (second score pair), K-major A operands
-        // K-major descriptor of k-step kk of an E-ring tile / of a shared-memory owner tensor: k-steps 0..3 lie
-        // in the 128-byte-swizzled atom, k-step 4 in the unswizzled block behind it
-        auto e_kdesc = [&](uint32_t tile, int kk) -> uint64_t {
-            return kk < 4 ? ptx::smem_desc_sw128(tile, 16, 1024) + (uint64_t)((kk * 32) >> 4)
-                          : ptx::smem_desc_nosw(tile + BC * 128, BC * 16, 128);
+        // Score MMAs: with the two tensors of a stage forming one K-major operand of 2 * BC rows,
+        //   [S | X0 Y1^T] = X0 [Y0 | Y1]^T is ONE N = 128 MMA per k-step and Sd += X1 Y0^T one N = 64 MMA:
+        // ten instructions per score pair instead of fifteen (an MMA costs its issuing warp 40 to 70 clocks
+        // next to the element-wise warps whatever its size), and the shared-memory port moves A once for both.
+        constexpr uint32_t idesc_s2 = ptx::idesc_bf16_f32(128, 2 * BC, 0, 0);
+        constexpr uint32_t HI_SW128 = ptx::desc_hi_sw128(1024), HI_TAIL = ptx::desc_hi_nosw(128);
+        // low descriptor halves (start address, leading offset); the high half is HI_SW128, or HI_TAIL for the
+        // unswizzled block that holds k-step 4 of tiles that are only read K-major
+        auto e_klo = [&](uint32_t stage, int kk) -> uint32_t {   // E stage, K-major, rows of Y0 (then Y1)
+            return kk < 4 ? ptx::desc_lo(stage, 16) + 2u * kk : ptx::desc_lo(stage + 2 * BC * 128, 2 * BC * 16);
         };
+        auto l_klo = [&](uint32_t stage, int kk) -> uint32_t {   // L stage, K-major, rows of Y0 (then Y1)
+            return ptx::desc_lo(stage + (kk >> 2) * 2 * BC * 128, 16) + 2u * (kk & 3);
+        };
+        auto own_klo = [&](uint32_t tile, int kk) -> uint32_t {  // shared-memory owner tile, K-major
+            return kk < 4 ? ptx::desc_lo(tile, 16) + 2u * kk : ptx::desc_lo(tile + BWD_ROWS * 128, BWD_ROWS * 16);
+        };
+        // L stage read MN-major by the output GEMMs (tensor t, k-step u of 16 stream rows): atoms of 64 d-columns
+        // are 2 * BC * 128 bytes apart, 8-row groups 1024 bytes apart
+        auto l_nlo = [&](uint32_t stage, int t, int u) -> uint32_t {
+            return ptx::desc_lo(stage + t * BC * 128, 2 * BC * 128) + (uint32_t)((u * 16 * 128) >> 4);
+        };
+        auto desc64 = [](uint32_t lo, uint32_t hi) -> uint64_t { return (static_cast<uint64_t>(hi) << 32) | lo; };
         // tiles this CTA streams over all of its items; tile g belongs to item g / T of this CTA
         const int n_it = (int)blockIdx.x < items ? (items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
         const int G = n_it * T;
@@ -690,17 +715,22 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             if (j < 2 && !ptx::mbar_wait_warp(bar(C::B_QREADY + (it & 1)), (it >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) return false;
             ptx::tc_fence_after_sync();
             // Y0, Y1 in the E ring, K-major B
-            const uint32_t t0 = tile_addr(0, g), t1 = tile_addr(1, g);
+            const uint32_t st = e_stage(g);
             const uint32_t dS = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, dT = dS + BC;
+            // (fifteen N = 64 MMAs: here, with every A operand in tensor memory and two issuers, the N = 128 form
+            // of the two-pair passes measured 4 to 6 % slower)
+            const uint32_t y1 = st + BC * 128, y1t = st + 2 * BC * 128 + BC * 16;  // rows of Y1: atom, tail block
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk)  // S = X0 Y0^T
-                ptx::mma_ts_elect(dS, ax0 + 8 * kk, e_kdesc(t0, kk), idesc_s, kk > 0 ? 1u : 0u);
+                ptx::mma_ts_elect(dS, ax0 + 8 * kk, desc64(e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk)  // Sd = X1 Y0^T
-                ptx::mma_ts_elect(dT, ax1 + 8 * kk, e_kdesc(t0, kk), idesc_s, kk > 0 ? 1u : 0u);
+                ptx::mma_ts_elect(dT, ax1 + 8 * kk, desc64(e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk)  // Sd += X0 Y1^T
-                ptx::mma_ts_elect(dT, ax0 + 8 * kk, e_kdesc(t1, kk), idesc_s, 1u);
+                ptx::mma_ts_elect(dT, ax0 + 8 * kk,
+                                  kk < 4 ? desc64(ptx::desc_lo(y1, 16) + 2u * kk, HI_SW128) : desc64(ptx::desc_lo(y1t, 2 * BC * 16), HI_TAIL),
+                                  idesc_s, 1u);
             ptx::mma_commit_elect(bar(C::B_SFULL + b));
             ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
             return true;
@@ -716,8 +746,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             ptx::tc_fence_after_sync();
             const uint32_t a0 = tb + C::COL_SCORE + b * C::SCORE_BUF_COLS, a1 = a0 + BC;
             // MN-major B (the L ring): atoms of 64 d-columns are BC*128 bytes apart, 8-row groups 1024 bytes apart
-            const uint64_t b0 = ptx::smem_desc_sw128(tile_addr(2, g), BC * 128, 1024);
-            const uint64_t b1 = ptx::smem_desc_sw128(tile_addr(3, g), BC * 128, 1024);
+            const uint64_t b0 = desc64(l_nlo(l_stage(g), 0, 0), HI_SW128);
+            const uint64_t b1 = desc64(l_nlo(l_stage(g), 1, 0), HI_SW128);
             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
 #pragma unroll
             for (int u = 0; u < BC / 16; ++u) {
@@ -770,54 +800,35 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 // shares its scheduler with four element-wise warps, and every instruction it saves per MMA shortens
                 // the chain second pair -> phase B -> outputs -> second pair.  (DV and the forward, whose chains
                 // are not bound by the issue, measured 2 to 4 % slower this way and keep the elected-lane form.)
-                constexpr uint32_t HI_SW = ptx::desc_hi_sw128(1024), HI_E4 = ptx::desc_hi_nosw(128);
-                // k-step kk of a K-major tile whose columns from 64 on sit in an unswizzled block behind the atom
-                auto klo = [&](uint32_t tile, int rows, int kk) -> uint32_t {
-                    return kk < 4 ? ptx::desc_lo(tile, 16) + 2u * kk : ptx::desc_lo(tile + rows * 128, rows * 16);
-                };
-                // S = X0 Y0^T, Sd = X1 Y0^T + X0 Y1^T; X0, X1 in shared memory, Y0, Y1 in the L ring, all K-major.
+                constexpr uint32_t HI_SW = HI_SW128;
+                // [S | X0 Y1^T] = X0 [Y0 | Y1]^T, Sd += X1 Y0^T; X0, X1 in shared memory, Y0, Y1 in the L ring, all K-major.
                 // `last`: the item's last tile; the shared-memory owner tiles are free once these MMAs are done
                 auto issue_first_pair = [&](int g, bool last) {
                     const uint32_t el = ptx::elect_one();
-                    const uint32_t y0 = ptx::desc_lo(tile_addr(2, g), 16), y1 = ptx::desc_lo(tile_addr(3, g), 16);
+                    const uint32_t st = l_stage(g);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
-                        const uint32_t off = (uint32_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        const uint32_t ahi = kk < 4 ? HI_SW : HI_E4;
-                        if (kk == 0) ptx::mma_ss_p<0>(el, dS, klo(own_base, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
-                        else ptx::mma_ss_p<1>(el, dS, klo(own_base, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
+                        const uint32_t ahi = kk < 4 ? HI_SW128 : HI_TAIL;
+                        if (kk == 0) ptx::mma_ss_p<0>(el, dS, own_klo(own_base, kk), ahi, l_klo(st, kk), HI_SW128, idesc_s2);
+                        else ptx::mma_ss_p<1>(el, dS, own_klo(own_base, kk), ahi, l_klo(st, kk), HI_SW128, idesc_s2);
                     }
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) {
-                        const uint32_t off = (uint32_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        const uint32_t ahi = kk < 4 ? HI_SW : HI_E4;
-                        if (kk == 0) ptx::mma_ss_p<0>(el, dT, klo(own_base + C::OWN_BYTES, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
-                        else ptx::mma_ss_p<1>(el, dT, klo(own_base + C::OWN_BYTES, BWD_ROWS, kk), ahi, y0 + off, HI_SW, idesc_s);
-                    }
-#pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) {
-                        const uint32_t off = (uint32_t)(((kk >> 2) * BC * 128 + (kk & 3) * 32) >> 4);
-                        ptx::mma_ss_p<1>(el, dT, klo(own_base, BWD_ROWS, kk), kk < 4 ? HI_SW : HI_E4, y1 + off, HI_SW, idesc_s);
-                    }
+                    for (int kk = 0; kk < KS; ++kk)
+                        ptx::mma_ss_p<1>(el, dT, own_klo(own_base + C::OWN_BYTES, kk), kk < 4 ? HI_SW128 : HI_TAIL, l_klo(st, kk), HI_SW128, idesc_s);
                     ptx::mma_commit_p(el, bar(C::B_SFULL + 0));
                     if (last) ptx::mma_commit_p(el, bar(C::B_OWNFREE));
                 };
-                // D = X2 Y2^T, X = X3 Y2^T + X2 Y3^T; X2, X3 in tensor memory, Y2, Y3 in the E ring
+                // [D | X2 Y3^T] = X2 [Y2 | Y3]^T, X += X3 Y2^T; X2, X3 in tensor memory, Y2, Y3 in the E ring
                 auto issue_second_pair = [&](int g) {
                     const uint32_t el = ptx::elect_one();
-                    const uint32_t t2 = tile_addr(0, g), t3 = tile_addr(1, g);
+                    const uint32_t st = e_stage(g);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
-                        if (kk == 0) ptx::mma_ts_p<0>(el, dD, ax0 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
-                        else ptx::mma_ts_p<1>(el, dD, ax0 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                        if (kk == 0) ptx::mma_ts_p<0>(el, dD, ax0 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s2);
+                        else ptx::mma_ts_p<1>(el, dD, ax0 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s2);
                     }
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) {
-                        if (kk == 0) ptx::mma_ts_p<0>(el, dX, ax1 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
-                        else ptx::mma_ts_p<1>(el, dX, ax1 + 8 * kk, klo(t2, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
-                    }
-#pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_p<1>(el, dX, ax0 + 8 * kk, klo(t3, BC, kk), kk < 4 ? HI_SW : HI_E4, idesc_s);
+                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_p<1>(el, dX, ax1 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s);
                     ptx::mma_commit_p(el, bar(C::B_SFULL + 1));
                     ptx::mma_commit_p(el, bar(C::B_EEMPTY + g % SE));
                 };
@@ -858,7 +869,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         ptx::tc_fence_after_sync();
                         {
                             const uint32_t el = ptx::elect_one();
-                            const uint32_t b0 = ptx::desc_lo(tile_addr(2, g), BC * 128), b1 = ptx::desc_lo(tile_addr(3, g), BC * 128);  // MN-major B
+                            const uint32_t b0 = l_nlo(l_stage(g), 0, 0), b1 = l_nlo(l_stage(g), 1, 0);  // MN-major B
                             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
 #pragma unroll
                             for (int u = 0; u < BC / 16; ++u) {
