@@ -28,11 +28,17 @@ METRIC = "attn_jvp_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# GEMMs each kernel executes by design (x 2*B*H*N^2*d FLOP each, true d)
+# GEMM units (2*B*H*N^2*d FLOP each, true d) each kernel EXECUTES by design.  The backward passes recompute
+# scores: together they execute 24 units for the 15 the method counts (3 recompute + 3 cotangent-score + 9 output).
 KERNEL_GEMMS = {"fwd": 6, "bwd_rowsums": 0, "bwd_dv": 6, "bwd_dk": 9, "bwd_dq": 9}
+BWD_CREDITED_GEMMS = 15
+BWD_TC = ("bwd_dv", "bwd_dk", "bwd_dq")
+# (B,H,N,d) tensors each kernel reads + writes once (its algorithmic HBM bytes, in units of one tensor)
+KERNEL_TENSORS = {"fwd": 8, "bwd_rowsums": 4, "bwd_dv": 8, "bwd_dk": 10, "bwd_dq": 10}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/jvp_fwd_bwd_kernels_dit512.md (that workload only; None for anything else)
-NCU_TRAFFIC_BYTES = {"dit512": {"fwd": 282.4e6, "bwd_dv": 280.7e6, "bwd_dk": 364.2e6, "bwd_dq": 364.1e6}}
+# profiles/jvp_fwd_bwd_kernels_dit512.md (that workload only; None for anything else, and None once a kernel
+# has changed since the capture)
+NCU_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -182,6 +188,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="dit512")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="full", choices=["full", "detach"],
+                    help="detach: backward without dtO (no gradient through tO; Sec. 5.3 'detach JVP'), 10*B*H*N^2*d FLOP")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     args = ap.parse_args()
@@ -209,6 +217,11 @@ def main():
 
     wl = inputs.WORKLOADS[args.workload]
     f_fwd, f_bwd = inputs.flops(wl.B, wl.H, wl.N, wl.d)
+    detach = args.variant == "detach"
+    if detach:  # standard attention backward: S recompute, dP, dV, dK, dQ = 5 GEMM units
+        f_bwd = f_bwd * 5.0 / 15.0
+        KERNEL_GEMMS.update({"bwd_dv": 4, "bwd_dk": 6, "bwd_dq": 7})   # what the three passes still execute
+        KERNEL_TENSORS.update({"bwd_rowsums": 2, "bwd_dv": 6, "bwd_dk": 8, "bwd_dq": 8})
     host = {k: v.to(torch.bfloat16).pin_memory() for k, v in inputs.make_inputs(wl).items()}
     x = {k: v.to(dev) for k, v in host.items()}
     shape = x["Q"].shape
@@ -222,8 +235,12 @@ def main():
         binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], out=(O, tO, lse, mu))
 
     def bwd():
-        binding.tvm_attn_jvp_bwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], O, tO, lse, mu, x["dO"], x["dtO"],
-                                 out=grads, workspace=ws)
+        if detach:
+            binding.tvm_attn_jvp_bwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], O, tO, lse, mu, x["dO"], None,
+                                     out=grads[:3] + (None, None, None), workspace=ws)
+        else:
+            binding.tvm_attn_jvp_bwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], O, tO, lse, mu, x["dO"], x["dtO"],
+                                     out=grads, workspace=ws)
 
     def step():
         fwd()
@@ -259,11 +276,18 @@ def main():
         sampler.start()
         sampler.wait_first()
         sampler.mark()
+    # The timed region is exactly `steps` steps between two events.  A short region (20 steps are 30 ms) gives the
+    # clock sampler a single sample, so the same region is measured `repeats` times in a row, until about half a
+    # second has passed, and the median region is reported; every region keeps its own barrier + synchronise.
     launches0 = binding.tvm_attn_launch_count()
-    ms_total = timed(step, args.steps)
+    regions = [timed(step, args.steps)]
     launches = binding.tvm_attn_launch_count() - launches0
-    ms_fwd = timed(fwd, args.steps)
-    ms_bwd = timed(bwd, args.steps)
+    budget_ms = 500.0
+    while sum(regions) < budget_ms and len(regions) < 64:
+        regions.append(timed(step, args.steps))
+    ms_total = statistics.median(regions)
+    ms_fwd = statistics.median([timed(fwd, args.steps) for _ in range(max(1, min(len(regions), 16)))])
+    ms_bwd = statistics.median([timed(bwd, args.steps) for _ in range(max(1, min(len(regions), 16)))])
     clocks = sampler.stop() if rank == 0 else None
     binding.tvm_attn_check_status()
 
@@ -281,14 +305,16 @@ def main():
     kernel_ms = {k: statistics.mean(v) for k, v in per_kernel.items() if v}
 
     # end to end: pinned host inputs -> device, forward + backward, results -> pinned host
-    host_out = {k: torch.empty(shape, dtype=torch.bfloat16).pin_memory() for k in ("O", "tO", "dQ", "dK", "dV", "dtQ", "dtK", "dtV")}
+    out_names = ("O", "tO", "dQ", "dK", "dV") + (() if detach else ("dtQ", "dtK", "dtV"))
+    in_names = tuple(k for k in inputs.NAMES if not (detach and k == "dtO"))
+    host_out = {k: torch.empty(shape, dtype=torch.bfloat16).pin_memory() for k in out_names}
     host_stats = {k: torch.empty(shape[:3], dtype=torch.float32).pin_memory() for k in ("lse", "mu")}
 
     def e2e_step():
-        for k in inputs.NAMES:
+        for k in in_names:
             x[k].copy_(host[k], non_blocking=True)
         step()
-        for k, t in zip(("O", "tO", "dQ", "dK", "dV", "dtQ", "dtK", "dtV"), (O, tO) + grads):
+        for k, t in zip(out_names, (O, tO) + grads):
             host_out[k].copy_(t, non_blocking=True)
         host_stats["lse"].copy_(lse, non_blocking=True)
         host_stats["mu"].copy_(mu, non_blocking=True)
@@ -298,7 +324,7 @@ def main():
         ms_e2e = timed(e2e_step, args.e2e_steps) / args.e2e_steps
     else:
         ms_e2e = None
-    h2d = sum(host[k].numel() * 2 for k in inputs.NAMES)
+    h2d = sum(host[k].numel() * 2 for k in in_names)
     d2h = sum(t.numel() * 2 for t in host_out.values()) + sum(t.numel() * 4 for t in host_stats.values())
     binding.tvm_attn_check_status()
 
@@ -313,28 +339,69 @@ def main():
     fwd_tf = f_fwd / (ms_fwd / args.steps * 1e-3) / 1e12
     bwd_tf = f_bwd / (ms_bwd / args.steps * 1e-3) / 1e12
     unit_flops = 2.0 * wl.B * wl.H * wl.N * wl.N * wl.d
-    top = max((k for k in kernel_ms if KERNEL_GEMMS[k] > 0), key=lambda k: kernel_ms[k])
-    achieved = KERNEL_GEMMS[top] * unit_flops / (kernel_ms[top] * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
+    tensor_bytes = 2.0 * wl.B * wl.H * wl.N * wl.d
     total_k = sum(kernel_ms.values())
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    sm_max = (clocks or {}).get("sm_max_mhz")
+    # Which measured peak the fractions are taken against: the burst figure when the GPU ran at (nearly) its
+    # maximum clock through the timed regions or they were short, the sustained one when it ran power-capped.
+    at_max_clock = bool(sm_mhz and sm_max and sm_mhz >= 0.97 * sm_max)
+    short_run = sum(regions) < 1000.0
+    use_burst = at_max_clock or (short_run and not sm_mhz)
+    peak = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
+    peak_note = "%s %s bf16 GEMM peak: median SM clock %s of %s MHz over %d timed regions (%.0f ms)" % (
+        peak_src, "burst" if use_burst else "sustained", sm_mhz, sm_max, len(regions), sum(regions))
+
+    def cycles(ms):  # device time in SM clocks at the sampled median clock: comparable between short and long runs
+        return None if not sm_mhz else ms * 1e-3 * sm_mhz * 1e6
+
+    def fracs(tf):
+        return {"frac_of_burst_peak": tf / peaks["bf16_tflops"], "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+                "frac_of_nominal": tf / NOMINAL_BF16_TFLOPS}
+
+    # the dominant kernels: the three tensor-core passes of the backward, taken together
+    tc_ms = sum(kernel_ms[k] for k in BWD_TC)
+    credited_units = 5 if detach else BWD_CREDITED_GEMMS
+    credited = credited_units * unit_flops / (tc_ms * 1e-3) / 1e12
+    executed = sum(KERNEL_GEMMS[k] for k in BWD_TC) * unit_flops / (tc_ms * 1e-3) / 1e12
+    tc_bytes = sum(KERNEL_TENSORS[k] for k in BWD_TC) * tensor_bytes
+    tc_gbs = tc_bytes / (tc_ms * 1e-3) / 1e9
+    # whole-step bounds: analytic FLOP against the tensor peak, compulsory bytes (every kernel's own tensors once)
+    # against the HBM peak; the larger fraction names the binding bound
+    step_bytes = sum(KERNEL_TENSORS[k] for k in kernel_ms) * tensor_bytes
+    step_tensor_frac = (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12 / peak
+    step_hbm_frac = step_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]
+    fwd_hbm_frac = KERNEL_TENSORS["fwd"] * tensor_bytes / (ms_fwd / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"]
+    traffic = NCU_TRAFFIC_BYTES.get(args.workload)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": args.workload, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "per_gpu": True,
+        "config": {"workload": args.workload, "variant": args.variant, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "per_gpu": True,
+                   "timed_regions": len(regions),
                    "l2": "16 resident tensors of %.0f MB each, larger than the 126 MB L2; no flush" % (x["Q"].numel() * 2 / 1e6)},
-        "fwd": {"tflops": fwd_tf, "ms": ms_fwd / args.steps, "frac_of_burst_peak": fwd_tf / peaks["bf16_tflops"],
-                "frac_of_sustained_peak": fwd_tf / peaks["bf16_tflops_sustained"], "frac_of_nominal": fwd_tf / NOMINAL_BF16_TFLOPS},
-        "bwd": {"tflops": bwd_tf, "ms": ms_bwd / args.steps, "frac_of_burst_peak": bwd_tf / peaks["bf16_tflops"],
-                "frac_of_sustained_peak": bwd_tf / peaks["bf16_tflops_sustained"], "frac_of_nominal": bwd_tf / NOMINAL_BF16_TFLOPS},
+        "fwd": dict({"tflops": fwd_tf, "ms": ms_fwd / args.steps, "cycles": cycles(ms_fwd / args.steps),
+                     "frac": fwd_tf / peak, "hbm_frac": fwd_hbm_frac}, **fracs(fwd_tf)),
+        "bwd": dict({"tflops": bwd_tf, "ms": ms_bwd / args.steps, "cycles": cycles(ms_bwd / args.steps),
+                     "frac": bwd_tf / peak}, **fracs(bwd_tf)),
         "frac_of_burst_peak": value / world / peaks["bf16_tflops"],
         "kernels_ms": kernel_ms,
+        "kernels_cycles": {k: cycles(v) for k, v in kernel_ms.items()},
         "kernels_share": {k: v / total_k for k, v in kernel_ms.items()},
-        "roofline": {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "peak_source": peak_src + " (sustained bf16 GEMM; kernel timed inside a long step)",
-                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
-                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get(top),
-                     "flops_per_launch": KERNEL_GEMMS[top] * unit_flops},
+        "kernels_executed_tflops": {k: KERNEL_GEMMS[k] * unit_flops / (v * 1e-3) / 1e12 for k, v in kernel_ms.items() if KERNEL_GEMMS[k]},
+        "roofline": {"bound": "tensor" if step_tensor_frac >= step_hbm_frac else "hbm",
+                     "kernel": "+".join(BWD_TC), "achieved": credited, "peak": peak, "unit": "TFLOP/s",
+                     "frac": credited / peak, "peak_source": peak_note,
+                     "achieved_executed": executed, "frac_executed": executed / peak,
+                     "note": "achieved = the method's own %d GEMM units of the backward / summed duration of the three "
+                             "tensor-core passes; achieved_executed counts the %d units they execute (scores recomputed per pass)"
+                             % (credited_units, sum(KERNEL_GEMMS[k] for k in BWD_TC)),
+                     "flops_per_launch": credited_units * unit_flops,
+                     "flops_executed_per_launch": sum(KERNEL_GEMMS[k] for k in BWD_TC) * unit_flops,
+                     "traffic": None if not traffic else sum(traffic[k] for k in BWD_TC),
+                     "hbm": {"achieved": tc_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": tc_gbs / peaks["hbm_gbs"],
+                             "bytes_per_launch": tc_bytes},
+                     "step": {"tensor_frac": step_tensor_frac, "hbm_frac": step_hbm_frac, "bytes": step_bytes}},
         "e2e": None if ms_e2e is None else {
             "value": world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

@@ -90,9 +90,14 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
  *     dV = P^T G + (P*Nn)^T Hc     dtV = P^T Hc
  *     dQ = alpha (dA K + W tK)     dtQ = alpha W K
  *     dK = alpha (dA^T Q + W^T tQ) dtK = alpha W^T Q
- *   in : Q, K, V, tQ, tK, tV and the forward's O, tO, lse, mu; dO, dtO (B,H,N,d) dtype, both
- *        required (non-NULL)
- *   out: dQ, dK, dV, dtQ, dtK, dtV (B,H,N,d) dtype
+ *   in : Q, K, V, tQ, tK, tV and the forward's O, tO, lse, mu; dO, dtO (B,H,N,d) dtype.
+ *        One of dO, dtO may be NULL and then counts as zero; it is never read and the work that only
+ *        it feeds is skipped.  dtO == NULL is the "detach JVP" setting of Sec. 5.3 (memory and runtime
+ *        table: no gradient flows through tO): what remains is the standard attention backward for dO.
+ *        dO == NULL leaves steps 1-6 of App. C alone.  Both NULL is TVM_ATTN_INVALID_ARG.  For
+ *        d > 80 both cotangents are required (TVM_ATTN_UNSUPPORTED otherwise).
+ *   out: dQ, dK, dV, dtQ, dtK, dtV (B,H,N,d) dtype.  With dtO == NULL the tangent gradients are
+ *        identically zero: dtQ, dtK, dtV may then be NULL, and those given are set to zero.
  *   workspace: device scratch of at least tvm_attn_jvp_workspace_bytes(p, 1) bytes, 16-byte
  *        aligned; contents on return are unspecified.  Calls sharing one workspace must not
  *        overlap on the device.

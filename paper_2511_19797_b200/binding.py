@@ -106,6 +106,11 @@ def _check_tensors(ref, tensors):
             raise ValueError("tensors must be contiguous CUDA tensors")
 
 
+def _ptr(t):
+    """Device address of a tensor, or a null pointer for None (an absent cotangent or an unwanted output)."""
+    return None if t is None else t.data_ptr()
+
+
 def _stream_ptr(stream):
     s = stream if stream is not None else torch.cuda.current_stream()
     return ctypes.c_void_p(s.cuda_stream)
@@ -139,9 +144,11 @@ def tvm_attn_jvp_fwd(Q, K, V, tQ, tK, tV, scale=0.0, flags=0, out=None, stream=N
 def tvm_attn_jvp_bwd(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, scale=0.0, flags=0, out=None, workspace=None,
                      stream=None):
     """Backward: returns (dQ, dK, dV, dtQ, dtK, dtV).  `workspace` is a uint8 CUDA tensor of at least
-    tvm_attn_jvp_workspace_bytes(...) bytes; one is allocated with torch when not given."""
+    tvm_attn_jvp_workspace_bytes(...) bytes; one is allocated with torch when not given.
+    dO or dtO may be None (a zero cotangent; dtO=None is the "detach JVP" setting).  With dtO=None the entries
+    dtQ, dtK, dtV of `out` may be None too; tensors given there come back zero."""
     lib = load()
-    _check_tensors(Q, (K, V, tQ, tK, tV, O, tO, dO, dtO))
+    _check_tensors(Q, tuple(t for t in (K, V, tQ, tK, tV, O, tO, dO, dtO) if t is not None))
     p = _params(Q, scale, flags)
     need = int(lib.tvm_attn_jvp_workspace_bytes(ctypes.byref(p), 1))
     if workspace is None:
@@ -150,7 +157,7 @@ def tvm_attn_jvp_bwd(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, scale=0.0, fl
     with torch.cuda.device(Q.device):
         rc = lib.tvm_attn_jvp_bwd(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
                                   tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
-                                  mu.data_ptr(), dO.data_ptr(), dtO.data_ptr(), *[o.data_ptr() for o in outs],
+                                  mu.data_ptr(), _ptr(dO), _ptr(dtO), *[_ptr(o) for o in outs],
                                   workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     if rc != 0:
         _raise("tvm_attn_jvp_bwd", rc)
@@ -164,12 +171,12 @@ def tvm_attn_jvp_bwd_noalloc(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, out, 
     C entry point behind it, allocates nothing.  B*H*N may not exceed NOALLOC_MAX_ROWS.  Calls that may overlap
     on the GPU race on the shared scratch; the first call on a device should come before any stream capture."""
     lib = load()
-    _check_tensors(Q, (K, V, tQ, tK, tV, O, tO, dO, dtO) + tuple(out))
+    _check_tensors(Q, tuple(t for t in (K, V, tQ, tK, tV, O, tO, dO, dtO) + tuple(out) if t is not None))
     p = _params(Q, scale, flags)
     with torch.cuda.device(Q.device):
         rc = lib.tvm_attn_jvp_bwd_noalloc(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
                                           tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
-                                          mu.data_ptr(), dO.data_ptr(), dtO.data_ptr(), *[o.data_ptr() for o in out],
+                                          mu.data_ptr(), _ptr(dO), _ptr(dtO), *[_ptr(o) for o in out],
                                           _stream_ptr(stream))
     if rc != 0:
         _raise("tvm_attn_jvp_bwd_noalloc", rc)

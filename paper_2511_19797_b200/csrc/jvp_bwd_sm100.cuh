@@ -69,7 +69,13 @@ struct BwdParams {
     const float* sig1;  // rowsum(dtO * O)
     const float* cvec;  // rowsum(dO * O) + rowsum(dtO * tO)
     int* status;        // device status word; non-zero makes the kernel a no-op
+    // Absent cotangents (a null dO or dtO means zero; Sec. 5.3 "detach JVP" is dtO absent): bit 0 = Hc (dtO),
+    // bit 1 = G (dO).  An absent tensor is never loaded; where an MMA still reads its tile (the N = 128 score
+    // MMA of DK) the tile's shared memory is zeroed once, where it is an owner operand (DQ) zeros are staged, and
+    // the MMAs whose result would be exactly zero are not issued.  out0 may be null when Hc is absent.
+    int absent;
 };
+enum : int { ABSENT_HC = 1, ABSENT_G = 2 };
 
 template <int MODE, int DP>
 struct BwdCfg {
@@ -120,7 +126,8 @@ struct BwdCfg {
     static constexpr int B_OWNER = B_QREADY + 2;
     static constexpr int B_ACCFREE = B_OWNER + 1;  // + (item & 1): the element-wise warps have read the item's accumulators
     static constexpr int B_OWNFREE = B_ACCFREE + 2;  // the MMAs that read the shared-memory owner tiles of an item are done
-    static constexpr int NBARS = B_OWNFREE + 1;
+    static constexpr int B_DRAIN = B_OWNFREE + 1;    // + issuer: used once, while winding down after a time-out
+    static constexpr int NBARS = B_DRAIN + 2;
     static_assert(NBARS <= 48, "barrier table too small");
     static constexpr int STATS_FLOATS = SL * 4 * 64;
     static constexpr int MISC_BYTES = 48 * 8 + 64 + STATS_FLOATS * 4;
@@ -184,10 +191,11 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             const int ch = slot + 4 * i;
             const bool second = ch >= KS;
             const int kk = second ? ch - KS : ch;
-            const __nv_bfloat16* src = p.own[C::XT0 + (second ? 1 : 0)] + grow_ * p.d + 16 * kk;
+            const __nv_bfloat16* own = p.own[C::XT0 + (second ? 1 : 0)];  // null: an absent cotangent, staged as zeros
+            const __nv_bfloat16* src = own + grow_ * p.d + 16 * kk;
             v[i][0] = v[i][1] = make_uint4(0, 0, 0, 0);
-            if (ch < 2 * KS && valid_ && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
-            if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
+            if (own && ch < 2 * KS && valid_ && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
+            if (own && ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
         }
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
@@ -377,11 +385,11 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     q1[c >> 1] = ptx::pack_bf16(__uint_as_float(x1[c]) * p.out_scale, __uint_as_float(x1[c + 1]) * p.out_scale);
                 }
                 if (row_valid) {
-                    *reinterpret_cast<uint4*>(p0 + 16 * ch) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
                     *reinterpret_cast<uint4*>(p1 + 16 * ch) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
-                    if (16 * ch + 8 < p.d) {
-                        *reinterpret_cast<uint4*>(p0 + 16 * ch + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
-                        *reinterpret_cast<uint4*>(p1 + 16 * ch + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
+                    if (16 * ch + 8 < p.d) *reinterpret_cast<uint4*>(p1 + 16 * ch + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
+                    if (p.out0) {  // null with Hc absent: acc0 was never written and its gradient is zero
+                        *reinterpret_cast<uint4*>(p0 + 16 * ch) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
+                        if (16 * ch + 8 < p.d) *reinterpret_cast<uint4*>(p0 + 16 * ch + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
                     }
                 }
             }
@@ -446,6 +454,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         ptx::mbar_init(bar(C::B_ACCFREE), 16);
         ptx::mbar_init(bar(C::B_ACCFREE + 1), 16);
         ptx::mbar_init(bar(C::B_OWNFREE), 1);
+        ptx::mbar_init(bar(C::B_DRAIN), 1);
+        ptx::mbar_init(bar(C::B_DRAIN + 1), 1);
         ptx::fence_mbar_init();
     }
     if (NA == 2) {
@@ -470,6 +480,22 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
             ptx::fence_proxy_async_smem();
         }
+    }
+    if (MODE == BWD_DK && p.absent) {
+        // DK reads both cotangent tiles of an E stage in one N = 128 MMA: the never-loaded one must read as zero
+        const int t = (p.absent & ABSENT_HC) ? 0 : 1;
+        for (int i = threadIdx.x; i < SE * BC * 8; i += BWD_THREADS) {  // the 64-column atoms, 16 bytes at a time
+            const int st = i / (BC * 8), r = i - st * (BC * 8);
+            *reinterpret_cast<uint4*>(smem + C::NOWN_SMEM * C::OWN_BYTES + st * 2 * C::EST_BYTES + t * BC * 128 + r * 16) = make_uint4(0, 0, 0, 0);
+        }
+        if (NA == 2) {
+            for (int i = threadIdx.x; i < SE * 2 * BC; i += BWD_THREADS) {  // both chunk blocks of the tail area
+                const int st = i / (2 * BC), k = (i / BC) & 1, r = i % BC;
+                *reinterpret_cast<uint4*>(smem + C::NOWN_SMEM * C::OWN_BYTES + st * 2 * C::EST_BYTES + 2 * BC * 128 + k * 2 * BC * 16 +
+                                          t * BC * 16 + r * 16) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        ptx::fence_proxy_async_smem();
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
@@ -512,6 +538,10 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const uint32_t ring_base = ring == 0 ? e_base : l_base;
             const __nv_bfloat16* base0 = p.strm[2 * ring];
             const __nv_bfloat16* base1 = p.strm[2 * ring + 1];
+            // the ring that streams the cotangents (Hc, G): L in DV, E in DK; an absent one is not loaded
+            constexpr bool COT = (MODE == BWD_DV && ring == 1) || (MODE == BWD_DK && ring == 0);
+            const bool has0 = !COT || !(p.absent & ABSENT_HC), has1 = !COT || !(p.absent & ABSENT_G);
+            const uint32_t tx_bytes = ((has0 ? 1 : 0) + (has1 ? 1 : 0)) * BC * 128;
             [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
             // Destination of chunk 0 of row `lane` behind the 64-column atom: the E ring keeps compact
             // 16-byte-per-row blocks (K-major operands only), the L ring a second 128-byte-swizzled atom.
@@ -598,9 +628,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     if (!ok) break;
                     const uint32_t stage = ring_base + s * 2 * TB;
                     if (lane == 0) {
-                        ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
-                        ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
-                        ptx::tma_load_3d(stage + BC * 128, map1, bar(b_full + s), 0, j * BC, bh);
+                        ptx::mbar_arrive_expect_tx(bar(b_full + s), tx_bytes);
+                        if (has0) ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
+                        if (has1) ptx::tma_load_3d(stage + BC * 128, map1, bar(b_full + s), 0, j * BC, bh);
                     }
                     if constexpr (HAS_CP) {
                         [[maybe_unused]] const int rows_left = p.N - j * BC;  // rows of this tile that exist
@@ -629,8 +659,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                     const bool v = lane + 32 * rp < rows_left;
                                     const uint32_t dst = stage + dst_lane +
                                                          (ring == 0 ? k * 2 * BC * 16 + rp * 32 * 16 : rp * 32 * 128 + ((k ^ sw) << 4));
-                                    ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
-                                    ptx::cp_async_16(dst + (ring == 0 ? BC * 16 : BC * 128), v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
+                                    if (has0) ptx::cp_async_16(dst, v ? src0 + rp * d32 + 8 * k : base0, v ? 16u : 0u);
+                                    if (has1) ptx::cp_async_16(dst + (ring == 0 ? BC * 16 : BC * 128), v ? src1 + rp * d32 + 8 * k : base1, v ? 16u : 0u);
                                 }
                             }
                         }
@@ -656,12 +686,23 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
             if (HAS_CP) {
                 ptx::cp_async_wait<0>();  // nothing of ours stays in flight
-                if (ok && pend_s >= 0) {
+                if (pend_s >= 0) {      // (also after a time-out: the drain below waits for these barriers)
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
                     if (ring == 0 && owner_pend && lane == 0) ptx::mbar_arrive(bar(C::B_OWNER));
                 }
+            }
+            if (!ok) {
+                // Winding down after a time-out: the TMA loads this warp started write into this block's shared
+                // memory and must have landed before the block exits.  The last S fills are the ones that may
+                // still be in flight: stages below s carry the phase of this pass over the ring, the others the one before.
+                for (int k = 0; k < S; ++k) {
+                    const bool cur = k < s;
+                    if (!cur && it == 0 && ph == 0) continue;  // never filled
+                    ptx::mbar_wait_drain(bar(b_full + k), (cur ? ph : ph ^ 1) & 1, ptx::DRAIN_LIMIT_NS);
+                }
+                if (ring == 0 && NPAIR == 2 && it > 0) ptx::mbar_wait_drain(bar(C::B_OWNER), (it - 1) & 1, ptx::DRAIN_LIMIT_NS);
             }
         };
         if (warp == 0) produce(std::integral_constant<int, 0>{});
@@ -749,13 +790,16 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const uint64_t b0 = desc64(l_nlo(l_stage(g), 0, 0), HI_SW128);
             const uint64_t b1 = desc64(l_nlo(l_stage(g), 1, 0), HI_SW128);
             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+            const bool hasH = !(p.absent & ABSENT_HC), hasG = !(p.absent & ABSENT_G);  // B0 = Hc, B1 = G
 #pragma unroll
             for (int u = 0; u < BC / 16; ++u) {
                 const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
                 const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                ptx::mma_ts_elect(acc0, a0 + 16 * u, b0 + off, idesc_o, acc);   // acc0 += A0 B0
-                ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc_o, acc);   // acc1 += A1 B0
-                ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, 1u);    // acc1 += A0 B1
+                if (hasH) {
+                    ptx::mma_ts_elect(acc0, a0 + 16 * u, b0 + off, idesc_o, acc);   // acc0 += A0 B0
+                    ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc_o, acc);   // acc1 += A1 B0
+                }
+                if (hasG) ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, hasH ? 1u : acc);  // acc1 += A0 B1
             }
             ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
@@ -827,8 +871,11 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         if (kk == 0) ptx::mma_ts_p<0>(el, dD, ax0 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s2);
                         else ptx::mma_ts_p<1>(el, dD, ax0 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s2);
                     }
+                    // X3 Y2^T is zero when either factor is an absent cotangent: DK has Y2 = Hc, DQ has X3 = G
+                    if (!(p.absent & (MODE == BWD_DK ? ABSENT_HC : ABSENT_G))) {
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_p<1>(el, dX, ax1 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s);
+                        for (int kk = 0; kk < KS; ++kk) ptx::mma_ts_p<1>(el, dX, ax1 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s);
+                    }
                     ptx::mma_commit_p(el, bar(C::B_SFULL + 1));
                     ptx::mma_commit_p(el, bar(C::B_EEMPTY + g % SE));
                 };
@@ -870,18 +917,20 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         {
                             const uint32_t el = ptx::elect_one();
                             const uint32_t b0 = l_nlo(l_stage(g), 0, 0), b1 = l_nlo(l_stage(g), 1, 0);  // MN-major B
+                            const bool hasW = !(p.absent & ABSENT_HC);
                             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
 #pragma unroll
                             for (int u = 0; u < BC / 16; ++u) {
                                 const uint32_t off = (uint32_t)((u * 16 * 128) >> 4);
+                                // with Hc absent W is exactly zero (D = 0 from zero operands, Sigma1 = 0): its MMAs are skipped
                                 if (u == 0 && j == 0) {
-                                    ptx::mma_ts_p<0>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    if (hasW) ptx::mma_ts_p<0>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
                                     ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
                                 } else {
-                                    ptx::mma_ts_p<1>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    if (hasW) ptx::mma_ts_p<1>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
                                     ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
                                 }
-                                ptx::mma_ts_p<1>(el, acc1, dD + 16 * u, b1 + off, HI_SW, idesc_o);
+                                if (hasW) ptx::mma_ts_p<1>(el, acc1, dD + 16 * u, b1 + off, HI_SW, idesc_o);
                             }
                             ptx::mma_commit_p(el, bar(C::B_LEMPTY + g % SL));
                             if (j == T - 1) ptx::mma_commit_p(el, bar(C::B_FINAL));
@@ -896,6 +945,11 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     }
 
     // ---------------------------------------------------------------------- teardown
+    if ((warp == 1 || warp == 3) && *abort_flag) {
+        // after a time-out: the MMAs this warp queued must be done before the tensor memory is given back
+        ptx::mma_commit_elect(bar(C::B_DRAIN + (warp >> 1)));
+        ptx::mbar_wait_drain(bar(C::B_DRAIN + (warp >> 1)), 0, ptx::DRAIN_LIMIT_NS);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {

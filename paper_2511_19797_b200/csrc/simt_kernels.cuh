@@ -41,12 +41,13 @@ __device__ __forceinline__ float warp_sum(float x) {
 
 // Copies `rows` rows of a (N, d) head starting at row r0 into shared memory with row pitch `pitch`
 // floats; rows at or beyond N are filled with zeros.
+// A null `tensor` (an absent cotangent) reads as zeros.
 template <typename T>
-__device__ __forceinline__ void load_rows(float* dst, const T* head, int r0, int rows, int N, int d, int pitch) {
+__device__ __forceinline__ void load_rows(float* dst, const T* tensor, size_t head_off, int r0, int rows, int N, int d, int pitch) {
     for (int idx = threadIdx.x; idx < rows * d; idx += SIMT_THREADS) {
         const int r = idx / d, c = idx - r * d;
         const int gr = r0 + r;
-        dst[r * pitch + c] = gr < N ? to_f32(head[(size_t)gr * d + c]) : 0.0f;
+        dst[r * pitch + c] = (tensor && gr < N) ? to_f32(tensor[head_off + (size_t)gr * d + c]) : 0.0f;
     }
 }
 
@@ -73,8 +74,8 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
     const int i0 = (blockIdx.x % tiles) * SIMT_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    load_rows(sq, Q + head, i0, SIMT_ROWS, N, d, d);
-    load_rows(stq, tQ + head, i0, SIMT_ROWS, N, d, d);
+    load_rows(sq, Q, head, i0, SIMT_ROWS, N, d, d);
+    load_rows(stq, tQ, head, i0, SIMT_ROWS, N, d, d);
 
     float m[SIMT_RPW], l[SIMT_RPW], mt[SIMT_RPW];
     float accO[SIMT_RPW][SIMT_MAXK], accR[SIMT_RPW][SIMT_MAXK];
@@ -87,10 +88,10 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
 
     for (int j0 = 0; j0 < N; j0 += SIMT_TILE) {
         __syncthreads();
-        load_rows(sk, K + head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stk, tK + head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(sv, V + head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stv, tV + head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sk, K, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stk, tK, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sv, V, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stv, tV, head, j0, SIMT_TILE, N, d, pitch);
         __syncthreads();
         const bool valid = j0 + lane < N;
 #pragma unroll
@@ -201,12 +202,15 @@ bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* _
     for (int u = 0; u < ROWSUM_UNROLL; ++u) {
         const long long row = row0 + (long long)u * rpw;
         act[u] = row < rows && c < cpr;
+        g[u] = h[u] = t[u] = make_uint4(0, 0, 0, 0);  // a null G or Hc (absent cotangent) counts as zeros
         if (act[u]) {
             const size_t off = (size_t)row * d + (size_t)c * VEC;
-            g[u] = __ldg(reinterpret_cast<const uint4*>(G + off));
-            h[u] = __ldg(reinterpret_cast<const uint4*>(Hc + off));
             o[u] = __ldg(reinterpret_cast<const uint4*>(O + off));
-            t[u] = __ldg(reinterpret_cast<const uint4*>(tO + off));
+            if (G) g[u] = __ldg(reinterpret_cast<const uint4*>(G + off));
+            if (Hc) {
+                h[u] = __ldg(reinterpret_cast<const uint4*>(Hc + off));
+                t[u] = __ldg(reinterpret_cast<const uint4*>(tO + off));
+            }
         }
     }
 #pragma unroll
@@ -266,10 +270,10 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
     const size_t srow = bh * N;
     const int i0 = (blockIdx.x % tiles) * SIMT_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    load_rows(sq, Q + head, i0, SIMT_ROWS, N, d, d);
-    load_rows(stq, tQ + head, i0, SIMT_ROWS, N, d, d);
-    load_rows(sg, G + head, i0, SIMT_ROWS, N, d, d);
-    load_rows(sh, Hc + head, i0, SIMT_ROWS, N, d, d);
+    load_rows(sq, Q, head, i0, SIMT_ROWS, N, d, d);
+    load_rows(stq, tQ, head, i0, SIMT_ROWS, N, d, d);
+    load_rows(sg, G, head, i0, SIMT_ROWS, N, d, d);
+    load_rows(sh, Hc, head, i0, SIMT_ROWS, N, d, d);
 
     float st_lse[SIMT_RPW], st_mu[SIMT_RPW], st_s1[SIMT_RPW], st_c[SIMT_RPW];
     float aQ[SIMT_RPW][SIMT_MAXK], aT[SIMT_RPW][SIMT_MAXK];
@@ -283,10 +287,10 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
     }
     for (int j0 = 0; j0 < N; j0 += SIMT_TILE) {
         __syncthreads();
-        load_rows(sk, K + head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stk, tK + head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(sv, V + head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stv, tV + head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sk, K, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stk, tK, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sv, V, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stv, tV, head, j0, SIMT_TILE, N, d, pitch);
         __syncthreads();
         const bool valid = j0 + lane < N;
 #pragma unroll
@@ -329,7 +333,7 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
             const int c = lane + 32 * k;
             if (c < d) {
                 from_f32(dQ + head + (size_t)i * d + c, alpha * aQ[r][k]);
-                from_f32(dtQ + head + (size_t)i * d + c, alpha * aT[r][k]);
+                if (dtQ) from_f32(dtQ + head + (size_t)i * d + c, alpha * aT[r][k]);
             }
         }
     }
@@ -363,10 +367,10 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
     const size_t srow = bh * N;
     const int j0 = (blockIdx.x % tiles) * SIMT_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    load_rows(sk, K + head, j0, SIMT_ROWS, N, d, d);
-    load_rows(stk, tK + head, j0, SIMT_ROWS, N, d, d);
-    load_rows(sv, V + head, j0, SIMT_ROWS, N, d, d);
-    load_rows(stv, tV + head, j0, SIMT_ROWS, N, d, d);
+    load_rows(sk, K, head, j0, SIMT_ROWS, N, d, d);
+    load_rows(stk, tK, head, j0, SIMT_ROWS, N, d, d);
+    load_rows(sv, V, head, j0, SIMT_ROWS, N, d, d);
+    load_rows(stv, tV, head, j0, SIMT_ROWS, N, d, d);
 
     float aK[SIMT_RPW][SIMT_MAXK], aTK[SIMT_RPW][SIMT_MAXK], aV[SIMT_RPW][SIMT_MAXK], aTV[SIMT_RPW][SIMT_MAXK];
 #pragma unroll
@@ -376,10 +380,10 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
 
     for (int i0 = 0; i0 < N; i0 += SIMT_TILE) {
         __syncthreads();
-        load_rows(sq, Q + head, i0, SIMT_TILE, N, d, pitch);
-        load_rows(stq, tQ + head, i0, SIMT_TILE, N, d, pitch);
-        load_rows(sg, G + head, i0, SIMT_TILE, N, d, pitch);
-        load_rows(sh, Hc + head, i0, SIMT_TILE, N, d, pitch);
+        load_rows(sq, Q, head, i0, SIMT_TILE, N, d, pitch);
+        load_rows(stq, tQ, head, i0, SIMT_TILE, N, d, pitch);
+        load_rows(sg, G, head, i0, SIMT_TILE, N, d, pitch);
+        load_rows(sh, Hc, head, i0, SIMT_TILE, N, d, pitch);
         __syncthreads();
         const bool valid = i0 + lane < N;
         const int i = min(i0 + lane, N - 1);
@@ -430,9 +434,9 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
             if (c < d) {
                 const size_t o = head + (size_t)j * d + c;
                 from_f32(dK + o, alpha * aK[r][k]);
-                from_f32(dtK + o, alpha * aTK[r][k]);
+                if (dtK) from_f32(dtK + o, alpha * aTK[r][k]);
                 from_f32(dV + o, aV[r][k]);
-                from_f32(dtV + o, aTV[r][k]);
+                if (dtV) from_f32(dtV + o, aTV[r][k]);
             }
         }
     }

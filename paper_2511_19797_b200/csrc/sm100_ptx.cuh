@@ -63,6 +63,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Wait used only while a block winds down after a time-out: polls until the phase completes or `limit_ns` have
+// passed, whatever the abort flag says.  Lets a role make sure that the asynchronous operations it started itself
+// (TMA loads into this block's shared memory, queued MMAs) have landed before the block frees its tensor memory
+// and exits.
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+    const uint64_t t0 = globaltimer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u && globaltimer_ns() - t0 > limit_ns) return false;
+    }
+}
+constexpr uint64_t DRAIN_LIMIT_NS = 2ull * 1000ull * 1000ull;
+
 // Orders generic-proxy shared-memory writes before later async-proxy (TMA / tcgen05) reads.
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

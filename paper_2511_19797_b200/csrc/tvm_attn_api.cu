@@ -237,13 +237,14 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
     using C = BwdCfg<MODE, DP>;
     CUtensorMap ms[4], mo[2];
     for (int t = 0; t < 4; ++t) {
-        const int rc = make_tmap(&ms[t], strm[t], s, C::BC);
+        // an absent cotangent (null) is never loaded: its map is built on a present tensor and stays unused
+        const int rc = make_tmap(&ms[t], strm[t] ? strm[t] : strm[t ^ 1], s, C::BC);
         if (rc != TVM_ATTN_OK) return rc;
         prm.strm[t] = static_cast<const __nv_bfloat16*>(strm[t]);
         prm.own[t] = static_cast<const __nv_bfloat16*>(own[t]);
     }
     for (int t = 0; t < 2; ++t) {
-        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? C::XS0 + t : t], s, BWD_ROWS);
+        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? C::XS0 + t : t], s, BWD_ROWS);  // never a cotangent
         if (rc != TVM_ATTN_OK) return rc;
     }
     auto kern = jvp_bwd_kernel<MODE, DP>;
@@ -410,9 +411,18 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     Shape s;
     int rc = check_params(p, &s);
     if (rc != TVM_ATTN_OK) return rc;
-    const void* ptrs[] = {Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, dQ, dK, dV, dtQ, dtK, dtV, workspace};
+    const void* ptrs[] = {Q, K, V, tQ, tK, tV, O, tO, lse, mu, dQ, dK, dV, workspace};
     for (const void* x : ptrs)
         if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
+    // A null cotangent means zero (dtO null = the "detach JVP" setting: no gradient through tO).  With dtO null the
+    // tangent gradients are identically zero and their outputs may be null too.
+    if (!dO && !dtO) return TVM_ATTN_INVALID_ARG;
+    const void* opt[] = {dO, dtO, dtQ, dtK, dtV};
+    for (const void* x : opt)
+        if (x && !aligned16(x)) return TVM_ATTN_INVALID_ARG;
+    if (dtO && (!dtQ || !dtK || !dtV)) return TVM_ATTN_INVALID_ARG;
+    const int absent = (dtO ? 0 : ABSENT_HC) | (dO ? 0 : ABSENT_G);
+    if (absent && !s.simt && s.dp > 80) return TVM_ATTN_UNSUPPORTED;  // head dims above 80 need both cotangents
     const size_t rows = (size_t)s.BH * (size_t)s.N;
     if (workspace_bytes < 3 * sizeof(float) * rows) return TVM_ATTN_WORKSPACE_TOO_SMALL;
     float* sig1 = static_cast<float*>(workspace);
@@ -420,6 +430,12 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     float* lse2 = cvec + rows;  // lse * log2(e)
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     g_prof.begin_call();
+    if (!dtO) {  // the tangent gradients of a call without dtO are zero: written here, by no kernel
+        const size_t bytes = rows * (size_t)s.d * (s.fp32 ? 4 : 2);
+        void* zero_out[] = {dtQ, dtK, dtV};
+        for (void* z : zero_out)
+            if (z && cudaMemsetAsync(z, 0, bytes, st) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+    }
     if (s.simt) {
         if (s.fp32) {
             rc = launch_rowsums<float>(s, dO, dtO, O, tO, lse, sig1, cvec, lse2, st);
@@ -441,10 +457,10 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         std::memset(&b, 0, sizeof b);
         b.N = s.N; b.d = s.d; b.BH = (int)s.BH;
         b.alpha = s.alpha; b.c2 = s.alpha * 1.4426950408889634f;
-        b.lse2 = lse2; b.mu = mu; b.sig1 = sig1; b.cvec = cvec; b.status = status;
+        b.lse2 = lse2; b.mu = mu; b.sig1 = sig1; b.cvec = cvec; b.status = status; b.absent = absent;
         {   // dtV = P^T Hc, dV = P^T G + (P*Nn)^T Hc : owner keys (K, tK); stream queries (Q, tQ | Hc, G)
             BwdParams q = b; q.out_scale = 1.0f;
-            q.out0 = static_cast<__nv_bfloat16*>(dtV); q.out1 = static_cast<__nv_bfloat16*>(dV);
+            q.out0 = dtO ? static_cast<__nv_bfloat16*>(dtV) : nullptr; q.out1 = static_cast<__nv_bfloat16*>(dV);
             const void* own[4] = {K, tK, K, tK};
             const void* strm[4] = {Q, tQ, dtO, dO};
             rc = launch_bwd_pass_dp<BWD_DV>(s, own, strm, q, st);
@@ -452,7 +468,7 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         }
         {   // dtK = alpha W^T Q, dK = alpha (dA^T Q + W^T tQ) : owner keys (K, tK, V, tV); stream (Hc, G | Q, tQ)
             BwdParams q = b; q.out_scale = s.alpha;
-            q.out0 = static_cast<__nv_bfloat16*>(dtK); q.out1 = static_cast<__nv_bfloat16*>(dK);
+            q.out0 = dtO ? static_cast<__nv_bfloat16*>(dtK) : nullptr; q.out1 = static_cast<__nv_bfloat16*>(dK);
             const void* own[4] = {K, tK, V, tV};
             const void* strm[4] = {dtO, dO, Q, tQ};
             rc = launch_bwd_pass_dp<BWD_DK>(s, own, strm, q, st);
@@ -460,7 +476,7 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         }
         {   // dtQ = alpha W K, dQ = alpha (dA K + W tK) : owner queries (Q, tQ, Hc, G); stream (V, tV | K, tK)
             BwdParams q = b; q.out_scale = s.alpha;
-            q.out0 = static_cast<__nv_bfloat16*>(dtQ); q.out1 = static_cast<__nv_bfloat16*>(dQ);
+            q.out0 = dtO ? static_cast<__nv_bfloat16*>(dtQ) : nullptr; q.out1 = static_cast<__nv_bfloat16*>(dQ);
             const void* own[4] = {Q, tQ, dtO, dO};
             const void* strm[4] = {V, tV, K, tK};
             rc = launch_bwd_pass_dp<BWD_DQ>(s, own, strm, q, st);

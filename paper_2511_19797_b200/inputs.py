@@ -24,7 +24,7 @@ WORKLOADS = {
     "dit512": Workload("dit512", 16, 16, 1024, 72, 2, 0.5, 0.0),
     "large": Workload("large", 2, 24, 4096, 128, 3, 0.5, 0.05),
 }
-for _n in (256, 1024, 4096, 16384):
+for _n in (256, 1024, 4096, 16384, 32768):  # 32768: the longest sequence of the paper's kernel table (App. C)
     WORKLOADS["sweep%d" % _n] = Workload("sweep%d" % _n, max(1, 65536 // _n), 16, _n, 64, 4, 0.5, 0.0)
 
 NAMES = ("Q", "K", "V", "tQ", "tK", "tV", "dO", "dtO")

@@ -21,10 +21,14 @@ def rel_err(got, ref):
     return float(np.abs(got - ref).max() / (scale if scale > 1e-12 else 1.0))
 
 
-def run_case(wl, oracle_heads=None, dtype=torch.bfloat16, flags=0, scale=0.0, device="cuda:0"):
+def run_case(wl, oracle_heads=None, dtype=torch.bfloat16, flags=0, scale=0.0, device="cuda:0", absent=None, noalloc=False):
     """Runs the whole workload on the GPU and the oracle on `oracle_heads` (flat b*H+h indices; all
-    heads when None).  Returns ({name: rel_err}, gpu outputs, oracle outputs) over the compared heads."""
+    heads when None).  Returns ({name: rel_err}, gpu outputs, oracle outputs) over the compared heads.
+    absent: "dO" or "dtO" -- that cotangent is passed to the library as a null pointer and to the oracle as zeros.
+    noalloc: the backward goes through tvm_attn_jvp_bwd_noalloc (scratch inside the library)."""
     x = inputs.make_inputs(wl)
+    if absent is not None:
+        x[absent] = torch.zeros_like(x[absent])
     xr = {k: v.to(dtype) for k, v in x.items()}                      # what the GPU consumes
     B, H, N, d = xr["Q"].shape
     sel = None if oracle_heads is None else torch.as_tensor(list(oracle_heads), dtype=torch.long)
@@ -39,8 +43,14 @@ def run_case(wl, oracle_heads=None, dtype=torch.bfloat16, flags=0, scale=0.0, de
     dev = {k: v.to(device) for k, v in xr.items()}
     O, tO, lse, mu = binding.tvm_attn_jvp_fwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"],
                                               scale=scale, flags=flags)
-    grads = binding.tvm_attn_jvp_bwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"], O, tO, lse, mu,
-                                     dev["dO"], dev["dtO"], scale=scale, flags=flags)
+    if noalloc:
+        grads = binding.tvm_attn_jvp_bwd_noalloc(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"], O, tO, lse, mu,
+                                                 dev["dO"], dev["dtO"], out=tuple(torch.empty_like(O) for _ in range(6)),
+                                                 scale=scale, flags=flags)
+    else:
+        grads = binding.tvm_attn_jvp_bwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"], O, tO, lse, mu,
+                                         None if absent == "dO" else dev["dO"], None if absent == "dtO" else dev["dtO"],
+                                         scale=scale, flags=flags)
     binding.tvm_attn_check_status()
     got = dict(zip(FWD_NAMES + BWD_NAMES, [pick(t.float().cpu()).numpy() for t in (O, tO, lse, mu) + tuple(grads)]))
     rf = c_oracle.attn_jvp_fwd(*xo[:6], alpha)[:4]

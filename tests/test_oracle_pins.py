@@ -332,3 +332,26 @@ def test_numpy_oracle_accepts_a_subset_of_query_rows():
     part_b = onp.attn_jvp_bwd(sub(Q), K, V, sub(tQ), tK, tV, sub(G), sub(Hc), 0.37)
     _close(part_b[0], full_b[0][:, :, rows], 1e-14)
     _close(part_b[3], full_b[3][:, :, rows], 1e-14)
+
+
+@pytest.mark.parametrize("bwd", BWDS)
+def test_query_rows_with_zero_cotangents_contribute_nothing(bwd):
+    """A query row whose cotangents dO and dtO are zero adds nothing to any key-side gradient (every term of
+    App. C steps 2, 4 and 6 carries a factor from that row of the cotangents) and gets zero dQ, dtQ.  So the
+    key-side gradients of a problem whose cotangents live on a few rows are those of the few-row problem:
+    the GPU test at S = 32,768 relies on this to check every element of dK, dtK, dV, dtV."""
+    xs = _inputs(1, 2, 29, 8, seed=13)
+    rows = [2, 11, 28]
+    mask = np.zeros((1, 1, 29, 1))
+    mask[:, :, rows] = 1.0
+    Q, K, V, tQ, tK, tV, G, Hc = xs
+    G, Hc = G * mask, Hc * mask
+    full = bwd(Q, K, V, tQ, tK, tV, G, Hc, 0.41)
+    sub = lambda a: np.ascontiguousarray(a[:, :, rows])
+    part = onp.attn_jvp_bwd(sub(Q), K, V, sub(tQ), tK, tV, sub(G), sub(Hc), 0.41)
+    for i in (1, 2, 4, 5):                      # dK, dV, dtK, dtV
+        _close(part[i], full[i], 1e-13)
+    others = [i for i in range(29) if i not in rows]
+    for i in (0, 3):                            # dQ, dtQ
+        _close(part[i], full[i][:, :, rows], 1e-13)
+        assert not np.any(full[i][:, :, others])

@@ -249,3 +249,113 @@ def test_two_host_threads_on_two_streams():
     for i in range(2):
         for a, b in zip(results[i], serial[i]):
             assert torch.equal(a, b)
+
+
+def _sampled_query_rows(N, rows, seed):
+    """Query-side outputs of a B=1, H=2, d=64 problem with N keys on sampled query rows against the numpy oracle."""
+    from oracle import attn_jvp_numpy as onp
+    from tests._parity import rel_err
+    wl = inputs.custom(1, 2, N, 64, seed=seed, tangent_std=0.5)
+    x = {k: v.to(torch.bfloat16) for k, v in inputs.make_inputs(wl).items()}
+    dev = {k: v.cuda() for k, v in x.items()}
+    O, tO, lse, mu = binding.tvm_attn_jvp_fwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"])
+    grads = binding.tvm_attn_jvp_bwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"], O, tO, lse, mu,
+                                     dev["dO"], dev["dtO"])
+    binding.tvm_attn_check_status()
+    f64 = {k: v.to(torch.float64).numpy() for k, v in x.items()}
+    sub = lambda k: np.ascontiguousarray(f64[k][:, :, rows])
+    alpha = inputs.default_scale(64)
+    rO, rtO, rlse, rmu = onp.attn_jvp_fwd(sub("Q"), f64["K"], f64["V"], sub("tQ"), f64["tK"], f64["tV"], alpha)
+    rdQ, _, _, rdtQ, _, _ = onp.attn_jvp_bwd(sub("Q"), f64["K"], f64["V"], sub("tQ"), f64["tK"], f64["tV"], sub("dO"),
+                                             sub("dtO"), alpha)
+    pick = lambda t: t.float().cpu().numpy()[:, :, rows]
+    return {"O": rel_err(pick(O), rO), "tO": rel_err(pick(tO), rtO), "lse": rel_err(pick(lse), rlse),
+            "mu": rel_err(pick(mu), rmu), "dQ": rel_err(pick(grads[0]), rdQ), "dtQ": rel_err(pick(grads[3]), rdtQ)}
+
+
+def test_sequence_of_32768_query_side_on_sampled_rows():
+    """The longest sequence of the paper's kernel table (App. C, S = 32,768) on one GPU: O, tO, lse, mu, dQ, dtQ
+    on sampled query rows."""
+    errs = _sampled_query_rows(32768, [0, 127, 128, 9999, 16384, 20000, 32767], seed=6)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+def test_sequence_of_32768_key_side_with_cotangents_on_few_rows():
+    """Key-side gradients at S = 32,768, every element of them: the cotangents are non-zero on 48 query rows only,
+    so only those rows contribute to dK, dtK, dV, dtV and the whole-matrix numpy oracle can compute them from the
+    48 rows against all 32,768 keys, while the GPU runs the full problem.  Query rows with a zero cotangent must
+    come out with exactly zero dQ and dtQ."""
+    from oracle import attn_jvp_numpy as onp
+    from tests._parity import rel_err
+    N = 32768
+    wl = inputs.custom(1, 2, N, 64, seed=8, tangent_std=0.5)
+    x = {k: v.to(torch.bfloat16) for k, v in inputs.make_inputs(wl).items()}
+    rows = sorted(set(int(i) for i in np.random.default_rng(5).integers(0, N, 48)) | {0, 63, 64, N - 1})
+    mask = torch.zeros(1, 1, N, 1, dtype=torch.bfloat16)
+    mask[:, :, rows] = 1
+    x["dO"] = x["dO"] * mask
+    x["dtO"] = x["dtO"] * mask
+    dev = {k: v.cuda() for k, v in x.items()}
+    O, tO, lse, mu = binding.tvm_attn_jvp_fwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"])
+    dQ, dK, dV, dtQ, dtK, dtV = binding.tvm_attn_jvp_bwd(dev["Q"], dev["K"], dev["V"], dev["tQ"], dev["tK"], dev["tV"], O, tO,
+                                                         lse, mu, dev["dO"], dev["dtO"])
+    binding.tvm_attn_check_status()
+    f64 = {k: v.to(torch.float64).numpy() for k, v in x.items()}
+    sub = lambda k: np.ascontiguousarray(f64[k][:, :, rows])
+    alpha = inputs.default_scale(64)
+    rdQ, rdK, rdV, rdtQ, rdtK, rdtV = onp.attn_jvp_bwd(sub("Q"), f64["K"], f64["V"], sub("tQ"), f64["tK"], f64["tV"],
+                                                       sub("dO"), sub("dtO"), alpha)
+    f = lambda t: t.float().cpu().numpy()
+    errs = {"dK": rel_err(f(dK), rdK), "dtK": rel_err(f(dtK), rdtK), "dV": rel_err(f(dV), rdV), "dtV": rel_err(f(dtV), rdtV),
+            "dQ": rel_err(f(dQ)[:, :, rows], rdQ), "dtQ": rel_err(f(dtQ)[:, :, rows], rdtQ)}
+    assert_within(errs, BF16_FWD, BF16_BWD)
+    others = np.setdiff1d(np.arange(N), rows)
+    assert not f(dQ)[:, :, others].any() and not f(dtQ)[:, :, others].any()
+
+
+ABSENT_SHAPES = [(2, 3, 200, 72), (1, 2, 129, 64), (3, 50, 192, 72), (1, 4, 333, 40), (2, 2, 64, 80)]
+
+
+@pytest.mark.parametrize("absent", ["dtO", "dO"])
+@pytest.mark.parametrize("B,H,N,d", ABSENT_SHAPES)
+def test_absent_cotangent_counts_as_zero(absent, B, H, N, d):
+    """A null dO or dtO (Sec. 5.3 "detach JVP": no gradient through tO) against the oracle fed a zero cotangent."""
+    wl = inputs.custom(B, H, N, d, seed=500 + N + d)
+    heads = None if B * H <= 12 else [0, 7, 77, B * H - 1]
+    errs, got, _ = run_case(wl, oracle_heads=heads, absent=absent)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+    if absent == "dtO":
+        for k in ("dtQ", "dtK", "dtV"):
+            assert not got[k].any(), k
+
+
+@pytest.mark.parametrize("absent", ["dtO", "dO"])
+def test_absent_cotangent_on_the_headline_shape(absent):
+    errs, _, _ = run_case("dit512", oracle_heads=[0, 85, 255], absent=absent)
+    assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
+
+
+@pytest.mark.parametrize("absent", ["dtO", "dO"])
+def test_absent_cotangent_fp32_validation_mode(absent):
+    errs, _, _ = run_case("tiny", dtype=torch.float32, absent=absent)
+    assert_within(errs, FP32_TOL, FP32_TOL)
+
+
+def test_detached_backward_needs_no_tangent_gradient_buffers():
+    """With dtO absent the outputs dtQ, dtK, dtV may be null; dQ, dK, dV are those of the call that is given them."""
+    wl = inputs.custom(2, 2, 200, 72, seed=21)
+    x = {k: v.to(torch.bfloat16).cuda() for k, v in inputs.make_inputs(wl).items()}
+    fw = binding.tvm_attn_jvp_fwd(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"])
+    args = (x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"]) + tuple(fw)
+    full = binding.tvm_attn_jvp_bwd(*args, x["dO"], None)
+    three = tuple(torch.empty_like(x["Q"]) for _ in range(3)) + (None, None, None)
+    part = binding.tvm_attn_jvp_bwd(*args, x["dO"], None, out=three)
+    binding.tvm_attn_check_status()
+    for a, b in zip(part[:3], full[:3]):
+        assert torch.equal(a, b)
+    with pytest.raises(binding.TvmAttnError) as e:        # both cotangents absent: nothing to differentiate
+        binding.tvm_attn_jvp_bwd(*args, None, None)
+    assert e.value.code == -1
+    with pytest.raises(binding.TvmAttnError) as e:        # dtO given: its gradients need somewhere to go
+        binding.tvm_attn_jvp_bwd(*args, x["dO"], x["dtO"], out=three)
+    assert e.value.code == -1
