@@ -141,23 +141,6 @@ struct BwdCfg {
     static_assert(COL_SCORE + NBUF * SCORE_BUF_COLS <= 512, "TMEM over-subscribed");
 };
 
-// One element of the backward element-wise stage.  s, ts (and d, x for DK/DQ) are the raw score
-// accumulators; lse2 = lse * log2(e); returns the two bf16-bound operand values.
-template <int MODE>
-__device__ __forceinline__ void bwd_element(const BwdParams& p, float s, float ts, float dd, float xx, float lse2,
-                                            float mu, float sg, float cv, float& a0, float& a1) {
-    const float P = ptx::ex2(fmaf(s, p.c2, -lse2));
-    const float Nn = fmaf(p.alpha, ts, -mu);
-    if (MODE == BWD_DV) {
-        a0 = P;
-        a1 = P * Nn;
-    } else {
-        const float W = P * (dd - sg);
-        a0 = W;
-        a1 = fmaf(P, xx - cv, W * Nn);
-    }
-}
-
 // Element-wise warps of the backward passes: `w` in 0..15.
 template <int MODE, int DP>
 __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tmem_base, uint32_t bar0,
