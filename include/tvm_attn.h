@@ -139,6 +139,39 @@ int tvm_attn_jvp_bwd_noalloc(const tvm_attn_params* p, const void* Q, const void
                              void* dK, void* dV, void* dtQ, void* dtK, void* dtV, void* cuda_stream);
 
 /*
+ * RMSNorm QK-normalisation with a tangent: the step in front of the attention in the paper's transformer
+ * (Sec. 4 "semi-Lipschitz control": RMSNorm as QK-norm with a learnable scale; App. "Lipschitzness of
+ * RMSNorm" gives the definition and the Jacobian).  Per row x of Q (and of K), with the row's tangent tx and
+ * a per-channel scale g of d floats shared by all rows:
+ *     r = sqrt(mean(x^2) + eps)      y = g * x / r      ty = g * (tx / r - x (x . tx) / (d r^3))
+ * (the paper prints the sum under the root without the square; its Jacobian is that of the squared form,
+ * which is what is computed).  One call normalises Q and K; its outputs are the Q, tQ, K, tK of
+ * tvm_attn_jvp_fwd.  Memory-bound streaming kernels: every tensor is read or written once.
+ *   in : Q, tQ, K, tK (B,H,N,d) dtype; gQ, gK: d floats each (device, 16-byte aligned); eps >= 0
+ *   out: Qn, tQn, Kn, tKn (B,H,N,d) dtype
+ */
+int tvm_qk_rmsnorm_jvp_fwd(const tvm_attn_params* p, float eps, const void* Q, const void* tQ, const void* K,
+                           const void* tK, const float* gQ, const float* gK, void* Qn, void* tQn, void* Kn,
+                           void* tKn, void* cuda_stream);
+
+/*
+ * Backward of tvm_qk_rmsnorm_jvp_fwd through both outputs: given the cotangents of Qn, tQn, Kn, tKn (what
+ * tvm_attn_jvp_bwd returns as dQ, dtQ, dK, dtK), the gradients of the un-normalised Q, tQ, K, tK and of the
+ * two scales.  With J = (I - u u^T / d) / r, u = x / r (the Jacobian of App. "Lipschitzness of RMSNorm"),
+ * a = g * dy, b = g * dty:
+ *     dtx = J b        dx = J a + d/dx [ b . (J(x) tx) ]        dg = sum over rows of dy * u + dty * (J tx)
+ * The normalised tensors are not needed: r is recomputed from x.  dgQ, dgK (d floats each) are written, not
+ * accumulated into, and are bit-reproducible (fixed summation order).
+ *   workspace: at least tvm_qk_rmsnorm_jvp_workspace_bytes(p) bytes of device scratch, 16-byte aligned
+ *        (partial sums of the scale gradients); 0 is returned for invalid parameters.
+ */
+size_t tvm_qk_rmsnorm_jvp_workspace_bytes(const tvm_attn_params* p);
+int tvm_qk_rmsnorm_jvp_bwd(const tvm_attn_params* p, float eps, const void* Q, const void* tQ, const void* K,
+                           const void* tK, const float* gQ, const float* gK, const void* dQn, const void* dtQn,
+                           const void* dKn, const void* dtKn, void* dQ, void* dtQ, void* dK, void* dtK,
+                           float* dgQ, float* dgK, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and reports what the kernels enqueued so far on the current device
  * recorded: TVM_ATTN_OK, TVM_ATTN_DEVICE_TIMEOUT if a bounded wait inside a tensor-core kernel gave
  * up (its outputs are then unspecified; the context stays usable), or TVM_ATTN_CUDA_ERROR.  Clears

@@ -34,6 +34,7 @@ class Params(ctypes.Structure):
 _lib = None
 EXPORTS = ("tvm_attn_jvp_workspace_bytes", "tvm_attn_jvp_fwd", "tvm_attn_jvp_bwd", "tvm_attn_jvp_bwd_noalloc",
            "tvm_attn_check_status", "tvm_attn_selftest_timeout",
+           "tvm_qk_rmsnorm_jvp_fwd", "tvm_qk_rmsnorm_jvp_bwd", "tvm_qk_rmsnorm_jvp_workspace_bytes",
            "tvm_attn_launch_count", "tvm_attn_strerror", "tvm_attn_version", "tvm_attn_set_profiling",
            "tvm_attn_get_profile")
 
@@ -65,6 +66,12 @@ def load(build_if_missing=False):
     lib.tvm_attn_jvp_bwd_noalloc.argtypes = [pp] + [vp] * 18 + [vp]
     lib.tvm_attn_check_status.restype = ctypes.c_int
     lib.tvm_attn_check_status.argtypes = [vp]
+    lib.tvm_qk_rmsnorm_jvp_workspace_bytes.restype = ctypes.c_size_t
+    lib.tvm_qk_rmsnorm_jvp_workspace_bytes.argtypes = [pp]
+    lib.tvm_qk_rmsnorm_jvp_fwd.restype = ctypes.c_int
+    lib.tvm_qk_rmsnorm_jvp_fwd.argtypes = [pp, ctypes.c_float] + [vp] * 10 + [vp]
+    lib.tvm_qk_rmsnorm_jvp_bwd.restype = ctypes.c_int
+    lib.tvm_qk_rmsnorm_jvp_bwd.argtypes = [pp, ctypes.c_float] + [vp] * 16 + [vp, ctypes.c_size_t, vp]
     lib.tvm_attn_selftest_timeout.restype = ctypes.c_int
     lib.tvm_attn_selftest_timeout.argtypes = [ctypes.c_uint64, vp]
     lib.tvm_attn_launch_count.restype = ctypes.c_uint64
@@ -181,6 +188,49 @@ def tvm_attn_jvp_bwd_noalloc(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, out, 
     if rc != 0:
         _raise("tvm_attn_jvp_bwd_noalloc", rc)
     return tuple(out)
+
+
+def _check_scale(g, ref):
+    if g.dtype != torch.float32 or g.dim() != 1 or g.numel() != ref.shape[-1] or g.device != ref.device or not g.is_contiguous():
+        raise ValueError("a scale must be a contiguous float32 CUDA vector of d elements")
+
+
+def tvm_qk_rmsnorm_jvp_fwd(Q, tQ, K, tK, gQ, gK, eps=1e-6, stream=None):
+    """RMSNorm QK-normalisation with a tangent: returns (Qn, tQn, Kn, tKn)."""
+    lib = load()
+    _check_tensors(Q, (tQ, K, tK))
+    _check_scale(gQ, Q)
+    _check_scale(gK, Q)
+    p = _params(Q, 0.0, 0)
+    outs = tuple(torch.empty_like(Q) for _ in range(4))
+    with torch.cuda.device(Q.device):
+        rc = lib.tvm_qk_rmsnorm_jvp_fwd(ctypes.byref(p), float(eps), Q.data_ptr(), tQ.data_ptr(), K.data_ptr(), tK.data_ptr(),
+                                        gQ.data_ptr(), gK.data_ptr(), *[o.data_ptr() for o in outs], _stream_ptr(stream))
+    if rc != 0:
+        _raise("tvm_qk_rmsnorm_jvp_fwd", rc)
+    return outs
+
+
+def tvm_qk_rmsnorm_jvp_bwd(Q, tQ, K, tK, gQ, gK, dQn, dtQn, dKn, dtKn, eps=1e-6, workspace=None, stream=None):
+    """Backward of the normalisation: returns (dQ, dtQ, dK, dtK, dgQ, dgK)."""
+    lib = load()
+    _check_tensors(Q, (tQ, K, tK, dQn, dtQn, dKn, dtKn))
+    _check_scale(gQ, Q)
+    _check_scale(gK, Q)
+    p = _params(Q, 0.0, 0)
+    need = int(lib.tvm_qk_rmsnorm_jvp_workspace_bytes(ctypes.byref(p)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=Q.device)
+    outs = tuple(torch.empty_like(Q) for _ in range(4))
+    dgQ, dgK = torch.empty_like(gQ), torch.empty_like(gK)
+    with torch.cuda.device(Q.device):
+        rc = lib.tvm_qk_rmsnorm_jvp_bwd(ctypes.byref(p), float(eps), Q.data_ptr(), tQ.data_ptr(), K.data_ptr(), tK.data_ptr(),
+                                        gQ.data_ptr(), gK.data_ptr(), dQn.data_ptr(), dtQn.data_ptr(), dKn.data_ptr(),
+                                        dtKn.data_ptr(), *[o.data_ptr() for o in outs], dgQ.data_ptr(), dgK.data_ptr(),
+                                        workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        _raise("tvm_qk_rmsnorm_jvp_bwd", rc)
+    return outs + (dgQ, dgK)
 
 
 def tvm_attn_check_status(stream=None, raise_on_error=True):

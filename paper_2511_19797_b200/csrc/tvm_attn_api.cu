@@ -14,6 +14,7 @@
 #include "dual_attn_sm100.cuh"
 #include "jvp_bwd_sm100.cuh"
 #include "jvp_fwd_sm100.cuh"
+#include "qk_rmsnorm.cuh"
 #include "simt_kernels.cuh"
 
 namespace tvm_attn {
@@ -347,6 +348,50 @@ __global__ void selftest_timeout_kernel(int* status, unsigned long long limit_ns
     if (!ok && threadIdx.x == 0 && abort_flag) atomicExch(status, 1);
 }
 
+// ------------------------------------------------------------------------------------------------
+// RMSNorm QK-normalisation prologue
+static int rms_geometry(const Shape& s, int* cpr, int* gs) {
+    *cpr = s.d * (s.fp32 ? 4 : 2) / 16;
+    int g = 1;
+    while (g < *cpr) g <<= 1;
+    *gs = g;
+    return g <= 32 ? TVM_ATTN_OK : TVM_ATTN_UNSUPPORTED;
+}
+
+template <typename T>
+static int rms_fwd(const Shape& s, float eps, const void* Q, const void* tQ, const void* K, const void* tK, const float* gQ,
+                   const float* gK, void* Qn, void* tQn, void* Kn, void* tKn, cudaStream_t st) {
+    int cpr, gs;
+    const int rc = rms_geometry(s, &cpr, &gs);
+    if (rc != TVM_ATTN_OK) return rc;
+    const long long rows = s.BH * s.N, rows_per_block = (long long)(RMS_THREADS / 32) * (32 / gs);
+    const RmsFwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (T*)Qn, (T*)tQn}, k{(const T*)K, (const T*)tK, gK, (T*)Kn, (T*)tKn};
+    const dim3 grid((unsigned)((rows + rows_per_block - 1) / rows_per_block), 2);
+    qk_rmsnorm_jvp_fwd_kernel<T><<<grid, RMS_THREADS, 0, st>>>(q, k, rows, s.d, cpr, gs, eps);
+    g_launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
+template <typename T>
+static int rms_bwd(const Shape& s, float eps, const void* Q, const void* tQ, const void* K, const void* tK, const float* gQ,
+                   const float* gK, const void* dQn, const void* dtQn, const void* dKn, const void* dtKn, void* dQ, void* dtQ,
+                   void* dK, void* dtK, float* dgQ, float* dgK, float* partial, cudaStream_t st) {
+    int cpr, gs;
+    const int rc = rms_geometry(s, &cpr, &gs);
+    if (rc != TVM_ATTN_OK) return rc;
+    const long long rows = s.BH * s.N;
+    float* pq = partial;
+    float* pk = partial + (size_t)RMS_BWD_BLOCKS * s.d;
+    const RmsBwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (const T*)dQn, (const T*)dtQn, (T*)dQ, (T*)dtQ, pq};
+    const RmsBwdSide<T> k{(const T*)K, (const T*)tK, gK, (const T*)dKn, (const T*)dtKn, (T*)dK, (T*)dtK, pk};
+    qk_rmsnorm_jvp_bwd_kernel<T><<<dim3(RMS_BWD_BLOCKS, 2), RMS_THREADS, 0, st>>>(q, k, rows, s.d, cpr, gs, eps);
+    qk_rmsnorm_dg_reduce_kernel<<<2, 128, 0, st>>>(pq, pk, dgQ, dgK, RMS_BWD_BLOCKS, s.d);
+    g_launches += 2;
+    return cuda_status(cudaGetLastError());
+}
+
+static bool rms_eps_ok(float eps) { return eps >= 0.0f && std::isfinite(eps); }
+
 }  // namespace tvm_attn
 
 using namespace tvm_attn;
@@ -533,6 +578,44 @@ int tvm_attn_check_status(void* cuda_stream) {
         return TVM_ATTN_DEVICE_TIMEOUT;
     }
     return TVM_ATTN_OK;
+}
+
+size_t tvm_qk_rmsnorm_jvp_workspace_bytes(const tvm_attn_params* p) {
+    Shape s;
+    if (check_params(p, &s) != TVM_ATTN_OK) return 0;
+    return (size_t)2 * RMS_BWD_BLOCKS * (size_t)s.d * sizeof(float);
+}
+
+int tvm_qk_rmsnorm_jvp_fwd(const tvm_attn_params* p, float eps, const void* Q, const void* tQ, const void* K, const void* tK,
+                           const float* gQ, const float* gK, void* Qn, void* tQn, void* Kn, void* tKn, void* cuda_stream) {
+    Shape s;
+    const int rc = check_params(p, &s);
+    if (rc != TVM_ATTN_OK) return rc;
+    if (!rms_eps_ok(eps)) return TVM_ATTN_INVALID_ARG;
+    const void* ptrs[] = {Q, tQ, K, tK, gQ, gK, Qn, tQn, Kn, tKn};
+    for (const void* x : ptrs)
+        if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    return s.fp32 ? rms_fwd<float>(s, eps, Q, tQ, K, tK, gQ, gK, Qn, tQn, Kn, tKn, st)
+                  : rms_fwd<__nv_bfloat16>(s, eps, Q, tQ, K, tK, gQ, gK, Qn, tQn, Kn, tKn, st);
+}
+
+int tvm_qk_rmsnorm_jvp_bwd(const tvm_attn_params* p, float eps, const void* Q, const void* tQ, const void* K, const void* tK,
+                           const float* gQ, const float* gK, const void* dQn, const void* dtQn, const void* dKn,
+                           const void* dtKn, void* dQ, void* dtQ, void* dK, void* dtK, float* dgQ, float* dgK, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+    Shape s;
+    const int rc = check_params(p, &s);
+    if (rc != TVM_ATTN_OK) return rc;
+    if (!rms_eps_ok(eps)) return TVM_ATTN_INVALID_ARG;
+    const void* ptrs[] = {Q, tQ, K, tK, gQ, gK, dQn, dtQn, dKn, dtKn, dQ, dtQ, dK, dtK, dgQ, dgK, workspace};
+    for (const void* x : ptrs)
+        if (!x || !aligned16(x)) return TVM_ATTN_INVALID_ARG;
+    if (workspace_bytes < (size_t)2 * RMS_BWD_BLOCKS * (size_t)s.d * sizeof(float)) return TVM_ATTN_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    float* part = static_cast<float*>(workspace);
+    return s.fp32 ? rms_bwd<float>(s, eps, Q, tQ, K, tK, gQ, gK, dQn, dtQn, dKn, dtKn, dQ, dtQ, dK, dtK, dgQ, dgK, part, st)
+                  : rms_bwd<__nv_bfloat16>(s, eps, Q, tQ, K, tK, gQ, gK, dQn, dtQn, dKn, dtKn, dQ, dtQ, dK, dtK, dgQ, dgK, part, st);
 }
 
 int tvm_attn_selftest_timeout(uint64_t limit_ns, void* cuda_stream) {

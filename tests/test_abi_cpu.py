@@ -20,7 +20,7 @@ def lib():
 def _declared_functions():
     text = open(os.path.join(ROOT, "include", "tvm_attn.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(tvm_attn_[a-z_0-9]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(tvm_(?:attn|qk)_[a-z_0-9]+)\s*\(", text)))
 
 
 def test_header_functions_are_all_exported(lib):
