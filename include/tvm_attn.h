@@ -8,9 +8,10 @@
  * differentiates through both outputs.
  *
  * Conventions for every entry point
- *   - All tensor pointers are DEVICE pointers on the current device, owned by the caller, packed
- *     (B, H, N, d) row-major (d contiguous) and 16-byte aligned.  Row statistics are (B, H, N)
- *     float.  The library never allocates, frees or keeps device memory.
+ *   - All tensor pointers are DEVICE pointers on the current device, owned by the caller, 16-byte
+ *     aligned, (B, H, rows, d) with d contiguous: packed by default, with the strides given in
+ *     tvm_attn_params otherwise.  Row statistics are packed (B, H, M) float.  The library never
+ *     allocates, frees or keeps device memory.
  *   - Outputs are fully overwritten, never accumulated into.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
  *     and the call returns without synchronising.
@@ -20,7 +21,7 @@
  *     be driven from one thread while it is enabled.
  *   - After a call returns, its results are complete for any work enqueued later on the same stream
  *     (plain stream order), although the kernels of one backward call overlap one another.
- *   - Self-attention, non-causal, no mask, bias or dropout: N queries attend to N keys per head.
+ *   - Non-causal, no mask, bias or dropout: M queries attend to N keys per head (M = N by default).
  */
 #ifndef TVM_ATTN_H_
 #define TVM_ATTN_H_
@@ -50,10 +51,21 @@ typedef enum {
 #define TVM_ATTN_FLAG_CUDA_CORES 1u /* run the CUDA-core validation kernels also for bf16 tensors   */
 
 typedef struct {
-    int32_t B, H, N, d; /* batch, heads, tokens (queries = keys), head dim; 8 <= d <= 128, d % 8 == 0 */
+    int32_t B, H, N, d; /* batch, heads, keys per head, head dim; 8 <= d <= 128, d % 8 == 0          */
     float scale;        /* softmax scale alpha of App. C; 0.0f selects 1/sqrt(d) with the true d     */
     int32_t dtype;      /* TVM_ATTN_BF16 or TVM_ATTN_FP32                                            */
     uint32_t flags;     /* 0 or TVM_ATTN_FLAG_*                                                      */
+    int32_t M;          /* queries per head (App. C "Background": Q in R^{M x d}, K, V in R^{N x d});
+                           0 = N, self-attention                                                      */
+    /* Element strides {row, head, batch} of the query-side tensors (Q, tQ, O, tO, dO, dtO, dQ, dtQ: M rows per
+       head) and of the key-side tensors (K, V, tK, tV, dK, dV, dtK, dtV: N rows per head).  All three zero selects
+       the packed layouts (B, H, M, d) and (B, H, N, d).  A (B, rows, H, d) tensor, or the Q, K, V slices of a
+       fused (B, rows, 3, H, d) projection read and written in place, are {row = H*d or 3*H*d, head = d,
+       batch = rows * row}.  The d elements of a row are contiguous; every stride is a multiple of 8 elements;
+       row >= d.  The statistics lse, mu and the workspace are always packed (B, H, M).  Strides and M != N
+       need d <= 80 (TVM_ATTN_UNSUPPORTED above). */
+    int64_t q_strides[3];
+    int64_t k_strides[3];
 } tvm_attn_params;
 
 /*

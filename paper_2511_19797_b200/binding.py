@@ -28,7 +28,8 @@ class TvmAttnError(RuntimeError):
 
 class Params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32), ("d", ctypes.c_int32),
-                ("scale", ctypes.c_float), ("dtype", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("scale", ctypes.c_float), ("dtype", ctypes.c_int32), ("flags", ctypes.c_uint32), ("M", ctypes.c_int32),
+                ("q_strides", ctypes.c_int64 * 3), ("k_strides", ctypes.c_int64 * 3)]
 
 
 _lib = None
@@ -92,25 +93,50 @@ def _raise(where, code):
     raise TvmAttnError(where, code, load().tvm_attn_strerror(code).decode())
 
 
-def _params(x, scale, flags):
-    if x.dim() != 4:
-        raise ValueError("expected (B, H, N, d) tensors")
-    if x.dtype == torch.bfloat16:
+def _strides(t):
+    """{row, head, batch} element strides of a (B, H, rows, d) tensor; zeros for the packed layout."""
+    if t.stride(3) != 1 and t.shape[3] != 1:
+        raise ValueError("the d elements of a row must be contiguous")
+    if t.is_contiguous():
+        return (0, 0, 0)
+    return (t.stride(2), t.stride(1), t.stride(0))
+
+
+def _params(q, scale, flags, k=None):
+    """Parameters from a query-side tensor q (B, H, M, d) and, for M != N or strided layouts, a key-side tensor k."""
+    if q.dim() != 4:
+        raise ValueError("expected (B, H, rows, d) tensors")
+    if q.dtype == torch.bfloat16:
         dt = BF16
-    elif x.dtype == torch.float32:
+    elif q.dtype == torch.float32:
         dt = FP32
     else:
         raise ValueError("tensors must be bfloat16 or float32")
-    B, H, N, d = x.shape
-    return Params(B, H, N, d, float(scale), dt, int(flags))
+    B, H, M, d = q.shape
+    k = q if k is None else k
+    if k.dim() != 4 or k.shape[0] != B or k.shape[1] != H or k.shape[3] != d:
+        raise ValueError("query-side and key-side tensors must agree in B, H and d")
+    N = k.shape[2]
+    p = Params(B, H, N, d, float(scale), dt, int(flags), 0 if M == N else M)
+    p.q_strides[:] = _strides(q)
+    p.k_strides[:] = _strides(k)
+    return p
 
 
 def _check_tensors(ref, tensors):
+    """Every tensor of one side shares shape, strides, dtype and device with the side's first tensor."""
     for t in tensors:
-        if t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device:
-            raise ValueError("all (B, H, N, d) tensors must share shape, dtype and device")
-        if not t.is_cuda or not t.is_contiguous():
-            raise ValueError("tensors must be contiguous CUDA tensors")
+        if t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device or t.stride() != ref.stride():
+            raise ValueError("all tensors of one side must share shape, strides, dtype and device")
+        if not t.is_cuda:
+            raise ValueError("tensors must be CUDA tensors")
+    if not ref.is_cuda:
+        raise ValueError("tensors must be CUDA tensors")
+
+
+def _like(t):
+    """A new tensor with the shape AND the strides of t (torch.empty_like does not keep the strides of a slice)."""
+    return torch.empty_strided(t.shape, t.stride(), dtype=t.dtype, device=t.device)
 
 
 def _ptr(t):
@@ -131,14 +157,15 @@ def tvm_attn_jvp_workspace_bytes(B, H, N, d, dtype=BF16, is_bwd=True, scale=0.0,
 def tvm_attn_jvp_fwd(Q, K, V, tQ, tK, tV, scale=0.0, flags=0, out=None, stream=None):
     """Forward: returns (O, tO, lse, mu).  `out` may hold preallocated (O, tO, lse, mu)."""
     lib = load()
-    _check_tensors(Q, (K, V, tQ, tK, tV))
-    p = _params(Q, scale, flags)
     if out is None:
-        O, tO = torch.empty_like(Q), torch.empty_like(Q)
+        O, tO = _like(Q), _like(Q)
         lse = torch.empty(Q.shape[:3], dtype=torch.float32, device=Q.device)
         mu = torch.empty_like(lse)
     else:
         O, tO, lse, mu = out
+    _check_tensors(Q, (tQ, O, tO))
+    _check_tensors(K, (V, tK, tV))
+    p = _params(Q, scale, flags, K)
     with torch.cuda.device(Q.device):
         rc = lib.tvm_attn_jvp_fwd(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
                                   tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
@@ -155,12 +182,13 @@ def tvm_attn_jvp_bwd(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, scale=0.0, fl
     dO or dtO may be None (a zero cotangent; dtO=None is the "detach JVP" setting).  With dtO=None the entries
     dtQ, dtK, dtV of `out` may be None too; tensors given there come back zero."""
     lib = load()
-    _check_tensors(Q, tuple(t for t in (K, V, tQ, tK, tV, O, tO, dO, dtO) if t is not None))
-    p = _params(Q, scale, flags)
+    p = _params(Q, scale, flags, K)
     need = int(lib.tvm_attn_jvp_workspace_bytes(ctypes.byref(p), 1))
     if workspace is None:
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=Q.device)
-    outs = out if out is not None else tuple(torch.empty_like(Q) for _ in range(6))
+    outs = out if out is not None else (_like(Q), _like(K), _like(K), _like(Q), _like(K), _like(K))
+    _check_tensors(Q, tuple(t for t in (tQ, O, tO, dO, dtO, outs[0], outs[3]) if t is not None))
+    _check_tensors(K, tuple(t for t in (V, tK, tV, outs[1], outs[2], outs[4], outs[5]) if t is not None))
     with torch.cuda.device(Q.device):
         rc = lib.tvm_attn_jvp_bwd(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
                                   tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
@@ -178,8 +206,9 @@ def tvm_attn_jvp_bwd_noalloc(Q, K, V, tQ, tK, tV, O, tO, lse, mu, dO, dtO, out, 
     C entry point behind it, allocates nothing.  B*H*N may not exceed NOALLOC_MAX_ROWS.  Calls that may overlap
     on the GPU race on the shared scratch; the first call on a device should come before any stream capture."""
     lib = load()
-    _check_tensors(Q, tuple(t for t in (K, V, tQ, tK, tV, O, tO, dO, dtO) + tuple(out) if t is not None))
-    p = _params(Q, scale, flags)
+    _check_tensors(Q, tuple(t for t in (tQ, O, tO, dO, dtO, out[0], out[3]) if t is not None))
+    _check_tensors(K, tuple(t for t in (V, tK, tV, out[1], out[2], out[4], out[5]) if t is not None))
+    p = _params(Q, scale, flags, K)
     with torch.cuda.device(Q.device):
         rc = lib.tvm_attn_jvp_bwd_noalloc(ctypes.byref(p), Q.data_ptr(), K.data_ptr(), V.data_ptr(), tQ.data_ptr(),
                                           tK.data_ptr(), tV.data_ptr(), O.data_ptr(), tO.data_ptr(), lse.data_ptr(),
@@ -198,11 +227,12 @@ def _check_scale(g, ref):
 def tvm_qk_rmsnorm_jvp_fwd(Q, tQ, K, tK, gQ, gK, eps=1e-6, stream=None):
     """RMSNorm QK-normalisation with a tangent: returns (Qn, tQn, Kn, tKn)."""
     lib = load()
-    _check_tensors(Q, (tQ, K, tK))
+    _check_tensors(Q, (tQ,))
+    _check_tensors(K, (tK,))
     _check_scale(gQ, Q)
     _check_scale(gK, Q)
-    p = _params(Q, 0.0, 0)
-    outs = tuple(torch.empty_like(Q) for _ in range(4))
+    p = _params(Q, 0.0, 0, K)
+    outs = (_like(Q), _like(Q), _like(K), _like(K))
     with torch.cuda.device(Q.device):
         rc = lib.tvm_qk_rmsnorm_jvp_fwd(ctypes.byref(p), float(eps), Q.data_ptr(), tQ.data_ptr(), K.data_ptr(), tK.data_ptr(),
                                         gQ.data_ptr(), gK.data_ptr(), *[o.data_ptr() for o in outs], _stream_ptr(stream))
@@ -214,14 +244,15 @@ def tvm_qk_rmsnorm_jvp_fwd(Q, tQ, K, tK, gQ, gK, eps=1e-6, stream=None):
 def tvm_qk_rmsnorm_jvp_bwd(Q, tQ, K, tK, gQ, gK, dQn, dtQn, dKn, dtKn, eps=1e-6, workspace=None, stream=None):
     """Backward of the normalisation: returns (dQ, dtQ, dK, dtK, dgQ, dgK)."""
     lib = load()
-    _check_tensors(Q, (tQ, K, tK, dQn, dtQn, dKn, dtKn))
+    _check_tensors(Q, (tQ, dQn, dtQn))
+    _check_tensors(K, (tK, dKn, dtKn))
     _check_scale(gQ, Q)
     _check_scale(gK, Q)
-    p = _params(Q, 0.0, 0)
+    p = _params(Q, 0.0, 0, K)
     need = int(lib.tvm_qk_rmsnorm_jvp_workspace_bytes(ctypes.byref(p)))
     if workspace is None:
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=Q.device)
-    outs = tuple(torch.empty_like(Q) for _ in range(4))
+    outs = (_like(Q), _like(Q), _like(K), _like(K))
     dgQ, dgK = torch.empty_like(gQ), torch.empty_like(gK)
     with torch.cuda.device(Q.device):
         rc = lib.tvm_qk_rmsnorm_jvp_bwd(ctypes.byref(p), float(eps), Q.data_ptr(), tQ.data_ptr(), K.data_ptr(), tK.data_ptr(),

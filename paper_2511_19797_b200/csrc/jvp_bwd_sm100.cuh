@@ -45,6 +45,7 @@
 #include <stdint.h>
 #include <type_traits>
 
+#include "geometry.cuh"
 #include "sm100_ptx.cuh"
 
 namespace tvm_attn {
@@ -56,7 +57,9 @@ constexpr int BWD_ROWS = 128;     // owner rows per CTA
 constexpr uint64_t BWD_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;
 
 struct BwdParams {
-    int N, d, BH;
+    int d, BH, H;
+    Geom o, s;    // owner side and stream side of this pass (DV, DK: keys own, queries stream; DQ: the other way round).
+                  // The per-query statistics are packed (B, H, M): indexed by stream rows in DV and DK, by owner rows in DQ.
     float alpha;      // softmax scale
     float c2;         // alpha * log2(e)
     float out_scale;  // factor applied to acc0 / acc1 in the epilogue
@@ -165,8 +168,8 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     auto stage_x = [&](int item, int item_index) {
         const int bh_ = item / row_tiles;
         const int row0_ = (item - bh_ * row_tiles) * BWD_ROWS;
-        const bool valid_ = row0_ + row < p.N;
-        const size_t grow_ = (size_t)bh_ * p.N + row0_ + row;
+        const bool valid_ = row0_ + row < p.o.rows;
+        const size_t ooff_ = p.o.head_off(bh_, p.H) + (size_t)(row0_ + row) * (size_t)p.o.rs;
         constexpr int NCH = (2 * KS + 3) / 4;  // chunks of 16 columns per warp, at most
         uint4 v[NCH][2];
 #pragma unroll
@@ -175,7 +178,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
             const bool second = ch >= KS;
             const int kk = second ? ch - KS : ch;
             const __nv_bfloat16* own = p.own[C::XT0 + (second ? 1 : 0)];  // null: an absent cotangent, staged as zeros
-            const __nv_bfloat16* src = own + grow_ * p.d + 16 * kk;
+            const __nv_bfloat16* src = own + ooff_ + 16 * kk;
             v[i][0] = v[i][1] = make_uint4(0, 0, 0, 0);
             if (own && ch < 2 * KS && valid_ && 16 * kk < p.d) v[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
             if (own && ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
@@ -203,8 +206,9 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         const int g0 = it * T;  // tiles this CTA has streamed before this item: rings and barrier phases run on
         const int bh = item / row_tiles;
         const int row0 = (item - bh * row_tiles) * BWD_ROWS;
-        const bool row_valid = row0 + row < p.N;
-        const size_t grow = (size_t)bh * p.N + row0 + row;
+        const bool row_valid = row0 + row < p.o.rows;
+        const size_t grow = (size_t)bh * p.o.rows + row0 + row;   // DQ: this query's slot in the packed statistics
+        const size_t ooff = p.o.head_off(bh, p.H) + (size_t)(row0 + row) * (size_t)p.o.rs;
         float r_lse2 = CUDART_INF_F, r_mu = 0.f, r_s1 = 0.f, r_cv = 0.f;  // per-row statistics (DQ)
         if (MODE == BWD_DQ && row_valid) {
             r_lse2 = p.lse2[grow];
@@ -296,7 +300,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                         } else {
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                lv[e] = (key0 + c4 + e < p.N) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
+                                lv[e] = (key0 + c4 + e < p.s.rows) ? r_lse2 : CUDART_INF_F;  // keys beyond N: P = 0
                                 mv[e] = r_mu; gv[e] = r_s1; cv[e] = r_cv;
                             }
                         }
@@ -354,8 +358,8 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         if (ok) ok = ptx::mbar_wait_warp(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
         if (ok) {
             ptx::tc_fence_after_sync();
-            __nv_bfloat16* p0 = p.out0 + grow * p.d;
-            __nv_bfloat16* p1 = p.out1 + grow * p.d;
+            __nv_bfloat16* p0 = p.out0 + ooff;
+            __nv_bfloat16* p1 = p.out1 + ooff;
             for (int ch = slot; ch < KS; ch += 4) {
                 uint32_t x0[16], x1[16];
                 ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, x0);
@@ -417,9 +421,9 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
     // per SM.  The rings, the score buffers and every barrier phase run on through the items (tile counter
     // g), so the loads, the operand staging and the first score MMAs of an item are under way while the
     // element-wise warps still write out the item before.
-    const int row_tiles = (p.N + BWD_ROWS - 1) / BWD_ROWS;
+    const int row_tiles = (p.o.rows + BWD_ROWS - 1) / BWD_ROWS;
     const int items = p.BH * row_tiles;
-    const int T = (p.N + BC - 1) / BC;  // stream tiles per item
+    const int T = (p.s.rows + BC - 1) / BC;  // stream tiles per item
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -506,7 +510,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
         // does not depend on the tile (lane's row, chunk positions, source pointers) is set up before it.
         constexpr int KT = NA == 2 ? (DP - 64) / 8 : 1;  // 16-byte chunks per row behind column 64, at most
         const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
-        const int d32 = 32 * p.d;                                      // 32 rows further down, in elements
+        const size_t d32 = 32 * (size_t)p.s.rs, d32o = 32 * (size_t)p.o.rs;  // 32 rows further down, in elements (stream, owner)
         bool owner_pend = false;  // owner-tile copies issued (warp 0) and not signalled yet
         auto produce = [&](auto ring_tag) -> void {
             constexpr int ring = decltype(ring_tag)::value;
@@ -525,13 +529,13 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             constexpr bool COT = (MODE == BWD_DV && ring == 1) || (MODE == BWD_DK && ring == 0);
             const bool has0 = !COT || !(p.absent & ABSENT_HC), has1 = !COT || !(p.absent & ABSENT_G);
             const uint32_t tx_bytes = ((has0 ? 1 : 0) + (has1 ? 1 : 0)) * BC * 128;
-            [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
+            [[maybe_unused]] const size_t tile_elems = (size_t)BC * (size_t)p.s.rs;
             // Destination of chunk 0 of row `lane` behind the 64-column atom: the E ring keeps compact
             // 16-byte-per-row blocks (K-major operands only), the L ring a second 128-byte-swizzled atom.
             [[maybe_unused]] const uint32_t dst_lane = 2 * BC * 128 + (ring == 0 ? lane * 16 : lane * 128);
             [[maybe_unused]] const uint32_t sw = lane & 7;  // rows 32 apart share it
             // statistics: 16-byte chunks when the rows of the (B, H, N) arrays are 16-byte aligned, else floats
-            const bool st16 = (p.N & 3) == 0;
+            const bool st16 = (p.s.rows & 3) == 0;
             [[maybe_unused]] const uint32_t st_base = ptx::smem_u32(stats);
             bool ok = true;
             int s = 0, ph = 0, pend_s = -1;  // pend_s: stage of the tile whose copied columns are not signalled yet
@@ -539,10 +543,12 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
                 const int bh = item / row_tiles;
                 [[maybe_unused]] const int row0 = (item - bh * row_tiles) * BWD_ROWS;
-                [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;  // element offset of (row `lane`, column 64)
+                const int cb = bh / p.H, chd = bh - cb * p.H;   // batch and head: coordinates of the 4-D tensor maps
+                // element offset of (row `lane`, column 64) in the stream tensors
+                [[maybe_unused]] const size_t lane_row = p.s.head_off(bh, p.H) + (size_t)lane * (size_t)p.s.rs + 64;
                 [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;  // advance by one tile per iteration
                 [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
-                [[maybe_unused]] const size_t srow = (size_t)bh * p.N;
+                [[maybe_unused]] const size_t srow = (size_t)bh * p.s.rows;
                 [[maybe_unused]] const float* st_src0 = (lane < 16 ? p.lse2 : p.mu) + srow + 4 * (lane & 15);
                 [[maybe_unused]] const float* st_src1 = NST == 4 ? (lane < 16 ? p.sig1 : p.cvec) + srow + 4 * (lane & 15) : nullptr;
                 if constexpr (ring == 0 && NPAIR == 2) {
@@ -568,13 +574,14 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     }
                     if (lane == 0) {
                         ptx::mbar_arrive_expect_tx(bar(C::B_OWNER), 2 * BWD_ROWS * 128);
-                        ptx::tma_load_3d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, bh);
-                        ptx::tma_load_3d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, bh);
+                        ptx::tma_load_4d(own_base, &tm_o2, bar(C::B_OWNER), 0, row0, chd, cb);
+                        ptx::tma_load_4d(own_base + C::OWN_BYTES, &tm_o3, bar(C::B_OWNER), 0, row0, chd, cb);
                     }
                     if constexpr (NA == 2) {
-                        const __nv_bfloat16* o2 = p.own[C::XS0] + lane_row + (size_t)row0 * p.d;
-                        const __nv_bfloat16* o3 = p.own[C::XS0 + 1] + lane_row + (size_t)row0 * p.d;
-                        const int rows_left = p.N - row0;
+                        const size_t lane_row_o = p.o.head_off(bh, p.H) + (size_t)(row0 + lane) * (size_t)p.o.rs + 64;
+                        const __nv_bfloat16* o2 = p.own[C::XS0] + lane_row_o;
+                        const __nv_bfloat16* o3 = p.own[C::XS0 + 1] + lane_row_o;
+                        const int rows_left = p.o.rows - row0;
 #pragma unroll
                         for (int k = 0; k < KT; ++k) {
                             if (k < ntail) {
@@ -582,8 +589,8 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                 for (int rp = 0; rp < BWD_ROWS / 32; ++rp) {
                                     const bool v = lane + 32 * rp < rows_left;
                                     const uint32_t dst = own_base + BWD_ROWS * 128 + k * BWD_ROWS * 16 + (lane + 32 * rp) * 16;
-                                    ptx::cp_async_16(dst, v ? o2 + rp * d32 + 8 * k : p.own[C::XS0], v ? 16u : 0u);
-                                    ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32 + 8 * k : p.own[C::XS0 + 1], v ? 16u : 0u);
+                                    ptx::cp_async_16(dst, v ? o2 + rp * d32o + 8 * k : p.own[C::XS0], v ? 16u : 0u);
+                                    ptx::cp_async_16(dst + C::OWN_BYTES, v ? o3 + rp * d32o + 8 * k : p.own[C::XS0 + 1], v ? 16u : 0u);
                                 }
                             }
                         }
@@ -612,11 +619,11 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     const uint32_t stage = ring_base + s * 2 * TB;
                     if (lane == 0) {
                         ptx::mbar_arrive_expect_tx(bar(b_full + s), tx_bytes);
-                        if (has0) ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
-                        if (has1) ptx::tma_load_3d(stage + BC * 128, map1, bar(b_full + s), 0, j * BC, bh);
+                        if (has0) ptx::tma_load_4d(stage, map0, bar(b_full + s), 0, j * BC, chd, cb);
+                        if (has1) ptx::tma_load_4d(stage + BC * 128, map1, bar(b_full + s), 0, j * BC, chd, cb);
                     }
                     if constexpr (HAS_CP) {
-                        [[maybe_unused]] const int rows_left = p.N - j * BC;  // rows of this tile that exist
+                        [[maybe_unused]] const int rows_left = p.s.rows - j * BC;  // rows of this tile that exist
                         if constexpr (STATS) {
                             // queries beyond N read as zero: their rows of the B operands are zero too
                             const uint32_t slot = st_base + s * (4 * 64 * 4);

@@ -41,6 +41,7 @@
 #include <math_constants.h>
 #include <stdint.h>
 
+#include "geometry.cuh"
 #include "sm100_ptx.cuh"
 
 namespace tvm_attn {
@@ -52,7 +53,8 @@ constexpr float FWD_LAZY_LOG2 = 3.0f;   // slack of the row reference, in log2 u
 constexpr uint64_t FWD_WAIT_LIMIT_NS = 200ull * 1000ull * 1000ull;
 
 struct FwdParams {
-    int N, d, BH;
+    int d, BH, H;
+    Geom q, k;    // query side (M rows per head: Q, tQ, O, tO) and key side (N rows: K, tK, V, tV)
     float alpha;  // softmax scale
     float c2;     // alpha * log2(e)
     const __nv_bfloat16* Q;
@@ -120,13 +122,13 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
     auto stage_q = [&](int item) {
         const int bh_ = item / row_tiles;
         const int row0_ = (item - bh_ * row_tiles) * FWD_ROWS;
-        const bool valid_ = row0_ + row < p.N;
-        const size_t grow_ = (size_t)bh_ * p.N + row0_ + row;
+        const bool valid_ = row0_ + row < p.q.rows;
+        const size_t qoff_ = p.q.head_off(bh_, p.H) + (size_t)(row0_ + row) * (size_t)p.q.rs;
         // the loads of the next chunk are in flight while this one is stored
         auto load = [&](int ch, uint4& v0, uint4& v1) {
             const bool is_t = ch >= KS;
             const int kk = is_t ? ch - KS : ch;
-            const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow_ * p.d + 16 * kk;
+            const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + qoff_ + 16 * kk;
             v0 = v1 = make_uint4(0, 0, 0, 0);
             if (ch < 2 * KS && valid_ && 16 * kk < p.d) v0 = __ldg(reinterpret_cast<const uint4*>(src));
             if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) v1 = __ldg(reinterpret_cast<const uint4*>(src + 8));
@@ -158,8 +160,9 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
     for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
         const int bh = item / row_tiles;
         const int row0 = (item - bh * row_tiles) * FWD_ROWS;
-        const bool row_valid = row0 + row < p.N;
-        const size_t grow = (size_t)bh * p.N + row0 + row;
+        const bool row_valid = row0 + row < p.q.rows;
+        const size_t grow = (size_t)bh * p.q.rows + row0 + row;   // the statistics are packed (B, H, M)
+        const size_t qoff = p.q.head_off(bh, p.H) + (size_t)(row0 + row) * (size_t)p.q.rs;
         float m_ref = -CUDART_INF_F, cen = 0.f;
         uint64_t l2 = 0ull, mt2 = 0ull;  // two partial sums each of P~ and of P~(T - c) over this warp's slices
 
@@ -172,7 +175,7 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             uint32_t s[16], ts[16];
             ptx::tmem_ld16(sbase + 16 * sl, s);
             ptx::tmem_wait_ld();
-            const int nvalid = p.N - j * BC - 16 * sl;  // columns of this slice that are real keys
+            const int nvalid = p.k.rows - j * BC - 16 * sl;  // columns of this slice that are real keys
             if (nvalid < 16) {
 #pragma unroll
                 for (int c = 0; c < 16; ++c)
@@ -295,14 +298,14 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             const int nitem = has_next ? item + (int)gridDim.x : item;
             const int bh_ = nitem / row_tiles;
             const int row0_ = (nitem - bh_ * row_tiles) * FWD_ROWS;
-            const bool valid_ = has_next && row0_ + row < p.N;
-            const size_t grow_ = (size_t)bh_ * p.N + row0_ + row;
+            const bool valid_ = has_next && row0_ + row < p.q.rows;
+            const size_t qoff_ = p.q.head_off(bh_, p.H) + (size_t)(row0_ + row) * (size_t)p.q.rs;
 #pragma unroll
             for (int i = 0; i < NCH; ++i) {
                 const int ch = sl + 4 * i;
                 const bool is_t = ch >= KS;
                 const int kk = is_t ? ch - KS : ch;
-                const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + grow_ * p.d + 16 * kk;
+                const __nv_bfloat16* src = (is_t ? p.tQ : p.Q) + qoff_ + 16 * kk;
                 nq[i][0] = nq[i][1] = make_uint4(0, 0, 0, 0);
                 if (ch < 2 * KS && valid_ && 16 * kk < p.d) nq[i][0] = __ldg(reinterpret_cast<const uint4*>(src));
                 if (ch < 2 * KS && valid_ && 16 * kk + 8 < p.d) nq[i][1] = __ldg(reinterpret_cast<const uint4*>(src + 8));
@@ -349,8 +352,8 @@ __device__ __forceinline__ void fwd_elementwise(const FwdParams& p, uint32_t tme
             }
             const float inv = 1.0f / l;
             const float mun = mt * inv;
-            __nv_bfloat16* o_ptr = p.O + grow * p.d;
-            __nv_bfloat16* t_ptr = p.tO + grow * p.d;
+            __nv_bfloat16* o_ptr = p.O + qoff;
+            __nv_bfloat16* t_ptr = p.tO + qoff;
             for (int ch = sl; ch < KS; ch += 4) {
                 uint32_t o[16], r[16];
                 ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, o);
@@ -408,9 +411,9 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // CTA per SM.  The rings, the score buffers and every barrier phase run on through the items (tile
     // counter g), so the loads and the first score MMAs of an item are under way while the element-wise
     // warps still write out the item before.
-    const int row_tiles = (p.N + FWD_ROWS - 1) / FWD_ROWS;
+    const int row_tiles = (p.q.rows + FWD_ROWS - 1) / FWD_ROWS;
     const int items = p.BH * row_tiles;
-    const int T = (p.N + BC - 1) / BC;  // key tiles per item
+    const int T = (p.k.rows + BC - 1) / BC;  // key tiles per item
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -475,15 +478,16 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const __nv_bfloat16* base0 = ring == 0 ? p.K : p.V;
         const __nv_bfloat16* base1 = ring == 0 ? p.tK : p.tV;
         [[maybe_unused]] const int ntail = NA == 2 ? (p.d - 64) >> 3 : 1;
-        [[maybe_unused]] const int d32 = 32 * p.d;
-        [[maybe_unused]] const size_t tile_elems = (size_t)BC * p.d;
+        [[maybe_unused]] const size_t d32 = 32 * (size_t)p.k.rs;             // 32 rows further down, in elements
+        [[maybe_unused]] const size_t tile_elems = (size_t)BC * (size_t)p.k.rs;
         [[maybe_unused]] const uint32_t dst_lane = BC * 128 + lane * 128;
         [[maybe_unused]] const uint32_t sw = lane & 7;
         bool ok = true;
         int s = 0, ph = 0, pend_s = -1;
         for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
             const int bh = item / row_tiles;
-            [[maybe_unused]] const size_t lane_row = ((size_t)bh * p.N + lane) * p.d + 64;
+            const int cb = bh / p.H, ch = bh - cb * p.H;   // batch and head: coordinates of the 4-D tensor maps
+            [[maybe_unused]] const size_t lane_row = p.k.head_off(bh, p.H) + (size_t)lane * (size_t)p.k.rs + 64;
             [[maybe_unused]] const __nv_bfloat16* src0 = base0 + lane_row;
             [[maybe_unused]] const __nv_bfloat16* src1 = base1 + lane_row;
             for (int j = 0; j < T; ++j) {
@@ -501,11 +505,11 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 const uint32_t stage = ring_base + s * 2 * TB;
                 if (lane == 0) {
                     ptx::mbar_arrive_expect_tx(bar(b_full + s), 2 * BC * 128);
-                    ptx::tma_load_3d(stage, map0, bar(b_full + s), 0, j * BC, bh);
-                    ptx::tma_load_3d(stage + TB, map1, bar(b_full + s), 0, j * BC, bh);
+                    ptx::tma_load_4d(stage, map0, bar(b_full + s), 0, j * BC, ch, cb);
+                    ptx::tma_load_4d(stage + TB, map1, bar(b_full + s), 0, j * BC, ch, cb);
                 }
                 if constexpr (NA == 2) {
-                    const int rows_left = p.N - j * BC;
+                    const int rows_left = p.k.rows - j * BC;
 #pragma unroll
                     for (int k = 0; k < KT; ++k) {
                         if (k < ntail) {

@@ -9,6 +9,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "geometry.cuh"
+
 namespace tvm_attn {
 
 constexpr int RMS_THREADS = 256;
@@ -64,22 +66,25 @@ __device__ __forceinline__ float rms_group_sum(float v, int gs) {
 template <typename T>
 struct RmsFwdSide {
     const T* x; const T* tx; const float* g; T* y; T* ty;
+    Geom geom;        // rows per head and strides of this side (Q: M rows, K: N rows)
+    long long rows;   // B * H * rows per head
 };
 
 // Forward for both sides (blockIdx.y = 0: Q, 1: K).  `cpr` = 16-byte chunks per row, `gs` = lanes per row.
 template <typename T>
 __global__ void __launch_bounds__(RMS_THREADS)
-qk_rmsnorm_jvp_fwd_kernel(const RmsFwdSide<T> q, const RmsFwdSide<T> k, long long rows, int d, int cpr, int gs, float eps) {
+qk_rmsnorm_jvp_fwd_kernel(const RmsFwdSide<T> q, const RmsFwdSide<T> k, int H, int d, int cpr, int gs, float eps) {
     constexpr int V = RmsVec<T>::N;
     const RmsFwdSide<T>& a = blockIdx.y == 0 ? q : k;
     const int lane = threadIdx.x & 31, rpw = 32 / gs;
     const int sub = lane / gs, c = lane - sub * gs;
     const long long row = ((long long)blockIdx.x * (RMS_THREADS / 32) + (threadIdx.x >> 5)) * rpw + sub;
-    const bool act = row < rows && c < cpr;
+    const bool act = row < a.rows && c < cpr;
     float x[V], t[V], g[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) x[i] = t[i] = g[i] = 0.f;
-    const size_t off = (size_t)row * d + (size_t)c * V;
+    const unsigned bh = (unsigned)row / (unsigned)a.geom.rows;   // rows fit 31 bits
+    const size_t off = a.geom.head_off((int)bh, H) + (size_t)((unsigned)row - bh * (unsigned)a.geom.rows) * (size_t)a.geom.rs + (size_t)c * V;
     if (act) {
         rms_load<T>(a.x + off, x);
         rms_load<T>(a.tx + off, t);
@@ -109,6 +114,8 @@ template <typename T>
 struct RmsBwdSide {
     const T* x; const T* tx; const float* g; const T* dy; const T* dty; T* dx; T* dtx;
     float* partial;   // [RMS_BWD_BLOCKS][d] partial sums of dg
+    Geom geom;
+    long long rows;
 };
 
 // Backward for both sides.  With a = g dy, b = g dty and the row sums ss = x.x, s = x.tx, ax = a.x, bx = b.x,
@@ -121,7 +128,7 @@ struct RmsBwdSide {
 // in a fixed order, so dg is bit-reproducible.
 template <typename T>
 __global__ void __launch_bounds__(RMS_THREADS)
-qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, long long rows, int d, int cpr, int gs, float eps) {
+qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, int H, int d, int cpr, int gs, float eps) {
     constexpr int V = RmsVec<T>::N;
     __shared__ float part[(RMS_THREADS / 32) * 32 * V];   // [warp][row in warp][column]; d * rows-per-warp <= 32 * V
     const RmsBwdSide<T>& a = blockIdx.y == 0 ? q : k;
@@ -133,13 +140,15 @@ qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, long lon
     for (int i = 0; i < V; ++i) g[i] = dg[i] = 0.f;
     if (c < cpr) rms_load_scale<V>(a.g + c * V, g);
     const float fd = (float)d;
+    const long long rows = a.rows;
     for (long long base = (long long)blockIdx.x * rows_per_block; base < rows; base += (long long)gridDim.x * rows_per_block) {
         const long long row = base + (long long)warp * rpw + sub;
         const bool act = row < rows && c < cpr;
         float x[V], t[V], gy[V], gt[V];
 #pragma unroll
         for (int i = 0; i < V; ++i) x[i] = t[i] = gy[i] = gt[i] = 0.f;
-        const size_t off = (size_t)row * d + (size_t)c * V;
+        const unsigned bh = (unsigned)row / (unsigned)a.geom.rows;   // rows fit 31 bits
+        const size_t off = a.geom.head_off((int)bh, H) + (size_t)((unsigned)row - bh * (unsigned)a.geom.rows) * (size_t)a.geom.rs + (size_t)c * V;
         if (act) {
             rms_load<T>(a.x + off, x);
             rms_load<T>(a.tx + off, t);

@@ -15,6 +15,8 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
+#include "geometry.cuh"
+
 namespace tvm_attn {
 
 constexpr int SIMT_ROWS = 16;
@@ -39,15 +41,15 @@ __device__ __forceinline__ float warp_sum(float x) {
     return x;
 }
 
-// Copies `rows` rows of a (N, d) head starting at row r0 into shared memory with row pitch `pitch`
-// floats; rows at or beyond N are filled with zeros.
+// Copies `rows` rows of a head (N rows of d elements, `rs` elements apart) starting at row r0 into shared memory
+// with row pitch `pitch` floats; rows at or beyond N are filled with zeros.
 // A null `tensor` (an absent cotangent) reads as zeros.
 template <typename T>
-__device__ __forceinline__ void load_rows(float* dst, const T* tensor, size_t head_off, int r0, int rows, int N, int d, int pitch) {
+__device__ __forceinline__ void load_rows(float* dst, const T* tensor, size_t head_off, long long rs, int r0, int rows, int N, int d, int pitch) {
     for (int idx = threadIdx.x; idx < rows * d; idx += SIMT_THREADS) {
         const int r = idx / d, c = idx - r * d;
         const int gr = r0 + r;
-        dst[r * pitch + c] = (tensor && gr < N) ? to_f32(tensor[head_off + (size_t)gr * d + c]) : 0.0f;
+        dst[r * pitch + c] = (tensor && gr < N) ? to_f32(tensor[head_off + (size_t)gr * rs + c]) : 0.0f;
     }
 }
 
@@ -58,7 +60,7 @@ __global__ void __launch_bounds__(SIMT_THREADS)
 simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __restrict__ V,
                 const T* __restrict__ tQ, const T* __restrict__ tK, const T* __restrict__ tV,
                 T* __restrict__ O, T* __restrict__ tO, float* __restrict__ lse, float* __restrict__ mu,
-                int N, int d, float alpha) {
+                Geom qg, Geom kg, int H, int d, float alpha) {
     extern __shared__ float smem[];
     const int pitch = d + 1;
     float* sq = smem;                       // [SIMT_ROWS][d]
@@ -68,14 +70,15 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
     float* sv = stk + SIMT_TILE * pitch;
     float* stv = sv + SIMT_TILE * pitch;
 
-    const int tiles = (N + SIMT_ROWS - 1) / SIMT_ROWS;
+    const int M = qg.rows, N = kg.rows;
+    const int tiles = (M + SIMT_ROWS - 1) / SIMT_ROWS;
     const size_t bh = blockIdx.x / tiles;
-    const size_t head = bh * N * d;
+    const size_t hq = qg.head_off((int)bh, H), hk = kg.head_off((int)bh, H);
     const int i0 = (blockIdx.x % tiles) * SIMT_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    load_rows(sq, Q, head, i0, SIMT_ROWS, N, d, d);
-    load_rows(stq, tQ, head, i0, SIMT_ROWS, N, d, d);
+    load_rows(sq, Q, hq, qg.rs, i0, SIMT_ROWS, M, d, d);
+    load_rows(stq, tQ, hq, qg.rs, i0, SIMT_ROWS, M, d, d);
 
     float m[SIMT_RPW], l[SIMT_RPW], mt[SIMT_RPW];
     float accO[SIMT_RPW][SIMT_MAXK], accR[SIMT_RPW][SIMT_MAXK];
@@ -88,10 +91,10 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
 
     for (int j0 = 0; j0 < N; j0 += SIMT_TILE) {
         __syncthreads();
-        load_rows(sk, K, head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stk, tK, head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(sv, V, head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stv, tV, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sk, K, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stk, tK, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sv, V, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stv, tV, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
         __syncthreads();
         const bool valid = j0 + lane < N;
 #pragma unroll
@@ -137,7 +140,7 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
 #pragma unroll
     for (int r = 0; r < SIMT_RPW; ++r) {
         const int i = i0 + warp * SIMT_RPW + r;
-        if (i >= N) continue;
+        if (i >= M) continue;
         const float inv = 1.0f / l[r];
         const float mun = mt[r] * inv;
 #pragma unroll
@@ -145,13 +148,13 @@ simt_fwd_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __res
             const int c = lane + 32 * k;
             if (c < d) {
                 const float o = accO[r][k] * inv;
-                from_f32(O + head + (size_t)i * d + c, o);
-                from_f32(tO + head + (size_t)i * d + c, fmaf(-mun, o, accR[r][k] * inv));
+                from_f32(O + hq + (size_t)i * qg.rs + c, o);
+                from_f32(tO + hq + (size_t)i * qg.rs + c, fmaf(-mun, o, accR[r][k] * inv));
             }
         }
         if (lane == 0) {
-            lse[bh * N + i] = m[r] + logf(l[r]);
-            mu[bh * N + i] = mun;
+            lse[bh * M + i] = m[r] + logf(l[r]);
+            mu[bh * M + i] = mun;
         }
     }
 }
@@ -189,7 +192,8 @@ template <typename T>
 __global__ void __launch_bounds__(ROWSUM_THREADS)
 bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* __restrict__ O,
                    const T* __restrict__ tO, const float* __restrict__ lse, float* __restrict__ sig1,
-                   float* __restrict__ cvec, float* __restrict__ lse2, long long rows, int d, int cpr, int gs) {
+                   float* __restrict__ cvec, float* __restrict__ lse2, long long rows, Geom qg, int H, int d, int cpr,
+                   int gs) {
     constexpr int VEC = 16 / (int)sizeof(T);
     const int lane = threadIdx.x & 31;
     const int rpw = 32 / gs;                  // rows per warp and step
@@ -204,7 +208,12 @@ bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* _
         act[u] = row < rows && c < cpr;
         g[u] = h[u] = t[u] = make_uint4(0, 0, 0, 0);  // a null G or Hc (absent cotangent) counts as zeros
         if (act[u]) {
-            const size_t off = (size_t)row * d + (size_t)c * VEC;
+            // the statistics are packed (B, H, M); the tensors have strides (H == 0 marks the packed layout: no division)
+            size_t off = (size_t)row * d + (size_t)c * VEC;
+            if (H > 0) {
+                const unsigned bh = (unsigned)row / (unsigned)qg.rows;   // rows fit 31 bits
+                off = qg.head_off((int)bh, H) + (size_t)((unsigned)row - bh * (unsigned)qg.rows) * (size_t)qg.rs + (size_t)c * VEC;
+            }
             o[u] = __ldg(reinterpret_cast<const uint4*>(O + off));
             if (G) g[u] = __ldg(reinterpret_cast<const uint4*>(G + off));
             if (Hc) {
@@ -230,6 +239,19 @@ bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* _
     }
 }
 
+// Writes zeros to every row of a tensor with strides (the gradients that are identically zero when a cotangent is
+// absent); 16 bytes per thread.
+__global__ void __launch_bounds__(256)
+zero_rows_kernel(uint4* __restrict__ t, Geom g, int H, long long rows, int chunks_per_row, int elems_per_chunk) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long row = idx / chunks_per_row;
+    if (row >= rows) return;
+    const int c = (int)(idx - row * chunks_per_row);
+    const unsigned bh = (unsigned)row / (unsigned)g.rows;   // rows fit 31 bits
+    const size_t off = g.head_off((int)bh, H) + (size_t)((unsigned)row - bh * (unsigned)g.rows) * (size_t)g.rs + (size_t)c * elems_per_chunk;
+    t[off / elems_per_chunk] = make_uint4(0, 0, 0, 0);   // every stride is a multiple of 16 bytes
+}
+
 // The four per-pair quantities of the backward from the six dot products of a (query, key) pair.
 struct PairTerms { float P, Pd, W, dA; };
 __device__ __forceinline__ PairTerms pair_terms(bool valid, float alpha, float s, float ts, float Dv, float X,
@@ -251,8 +273,8 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
                    const T* __restrict__ tQ, const T* __restrict__ tK, const T* __restrict__ tV,
                    const T* __restrict__ G, const T* __restrict__ Hc, const float* __restrict__ lse,
                    const float* __restrict__ mu, const float* __restrict__ sig1,
-                   const float* __restrict__ cvec, T* __restrict__ dQ, T* __restrict__ dtQ, int N, int d,
-                   float alpha) {
+                   const float* __restrict__ cvec, T* __restrict__ dQ, T* __restrict__ dtQ, Geom qg, Geom kg, int H,
+                   int d, float alpha) {
     extern __shared__ float smem[];
     const int pitch = d + 1;
     float* sq = smem;
@@ -264,22 +286,23 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
     float* sv = stk + SIMT_TILE * pitch;
     float* stv = sv + SIMT_TILE * pitch;
 
-    const int tiles = (N + SIMT_ROWS - 1) / SIMT_ROWS;
+    const int M = qg.rows, N = kg.rows;
+    const int tiles = (M + SIMT_ROWS - 1) / SIMT_ROWS;
     const size_t bh = blockIdx.x / tiles;
-    const size_t head = bh * N * d;
-    const size_t srow = bh * N;
+    const size_t hq = qg.head_off((int)bh, H), hk = kg.head_off((int)bh, H);
+    const size_t srow = bh * M;
     const int i0 = (blockIdx.x % tiles) * SIMT_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    load_rows(sq, Q, head, i0, SIMT_ROWS, N, d, d);
-    load_rows(stq, tQ, head, i0, SIMT_ROWS, N, d, d);
-    load_rows(sg, G, head, i0, SIMT_ROWS, N, d, d);
-    load_rows(sh, Hc, head, i0, SIMT_ROWS, N, d, d);
+    load_rows(sq, Q, hq, qg.rs, i0, SIMT_ROWS, M, d, d);
+    load_rows(stq, tQ, hq, qg.rs, i0, SIMT_ROWS, M, d, d);
+    load_rows(sg, G, hq, qg.rs, i0, SIMT_ROWS, M, d, d);
+    load_rows(sh, Hc, hq, qg.rs, i0, SIMT_ROWS, M, d, d);
 
     float st_lse[SIMT_RPW], st_mu[SIMT_RPW], st_s1[SIMT_RPW], st_c[SIMT_RPW];
     float aQ[SIMT_RPW][SIMT_MAXK], aT[SIMT_RPW][SIMT_MAXK];
 #pragma unroll
     for (int r = 0; r < SIMT_RPW; ++r) {
-        const int i = min(i0 + warp * SIMT_RPW + r, N - 1);
+        const int i = min(i0 + warp * SIMT_RPW + r, M - 1);
         st_lse[r] = lse[srow + i]; st_mu[r] = mu[srow + i];
         st_s1[r] = sig1[srow + i]; st_c[r] = cvec[srow + i];
 #pragma unroll
@@ -287,10 +310,10 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
     }
     for (int j0 = 0; j0 < N; j0 += SIMT_TILE) {
         __syncthreads();
-        load_rows(sk, K, head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stk, tK, head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(sv, V, head, j0, SIMT_TILE, N, d, pitch);
-        load_rows(stv, tV, head, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sk, K, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stk, tK, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
+        load_rows(sv, V, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
+        load_rows(stv, tV, hk, kg.rs, j0, SIMT_TILE, N, d, pitch);
         __syncthreads();
         const bool valid = j0 + lane < N;
 #pragma unroll
@@ -327,13 +350,13 @@ simt_bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __
 #pragma unroll
     for (int r = 0; r < SIMT_RPW; ++r) {
         const int i = i0 + warp * SIMT_RPW + r;
-        if (i >= N) continue;
+        if (i >= M) continue;
 #pragma unroll
         for (int k = 0; k < SIMT_MAXK; ++k) {
             const int c = lane + 32 * k;
             if (c < d) {
-                from_f32(dQ + head + (size_t)i * d + c, alpha * aQ[r][k]);
-                if (dtQ) from_f32(dtQ + head + (size_t)i * d + c, alpha * aT[r][k]);
+                from_f32(dQ + hq + (size_t)i * qg.rs + c, alpha * aQ[r][k]);
+                if (dtQ) from_f32(dtQ + hq + (size_t)i * qg.rs + c, alpha * aT[r][k]);
             }
         }
     }
@@ -349,7 +372,7 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
                     const T* __restrict__ G, const T* __restrict__ Hc, const float* __restrict__ lse,
                     const float* __restrict__ mu, const float* __restrict__ sig1,
                     const float* __restrict__ cvec, T* __restrict__ dK, T* __restrict__ dV,
-                    T* __restrict__ dtK, T* __restrict__ dtV, int N, int d, float alpha) {
+                    T* __restrict__ dtK, T* __restrict__ dtV, Geom qg, Geom kg, int H, int d, float alpha) {
     extern __shared__ float smem[];
     const int pitch = d + 1;
     float* sk = smem;
@@ -361,16 +384,17 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
     float* sg = stq + SIMT_TILE * pitch;
     float* sh = sg + SIMT_TILE * pitch;
 
+    const int M = qg.rows, N = kg.rows;
     const int tiles = (N + SIMT_ROWS - 1) / SIMT_ROWS;
     const size_t bh = blockIdx.x / tiles;
-    const size_t head = bh * N * d;
-    const size_t srow = bh * N;
+    const size_t hq = qg.head_off((int)bh, H), hk = kg.head_off((int)bh, H);
+    const size_t srow = bh * M;
     const int j0 = (blockIdx.x % tiles) * SIMT_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    load_rows(sk, K, head, j0, SIMT_ROWS, N, d, d);
-    load_rows(stk, tK, head, j0, SIMT_ROWS, N, d, d);
-    load_rows(sv, V, head, j0, SIMT_ROWS, N, d, d);
-    load_rows(stv, tV, head, j0, SIMT_ROWS, N, d, d);
+    load_rows(sk, K, hk, kg.rs, j0, SIMT_ROWS, N, d, d);
+    load_rows(stk, tK, hk, kg.rs, j0, SIMT_ROWS, N, d, d);
+    load_rows(sv, V, hk, kg.rs, j0, SIMT_ROWS, N, d, d);
+    load_rows(stv, tV, hk, kg.rs, j0, SIMT_ROWS, N, d, d);
 
     float aK[SIMT_RPW][SIMT_MAXK], aTK[SIMT_RPW][SIMT_MAXK], aV[SIMT_RPW][SIMT_MAXK], aTV[SIMT_RPW][SIMT_MAXK];
 #pragma unroll
@@ -378,15 +402,15 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
 #pragma unroll
         for (int k = 0; k < SIMT_MAXK; ++k) { aK[r][k] = 0.f; aTK[r][k] = 0.f; aV[r][k] = 0.f; aTV[r][k] = 0.f; }
 
-    for (int i0 = 0; i0 < N; i0 += SIMT_TILE) {
+    for (int i0 = 0; i0 < M; i0 += SIMT_TILE) {
         __syncthreads();
-        load_rows(sq, Q, head, i0, SIMT_TILE, N, d, pitch);
-        load_rows(stq, tQ, head, i0, SIMT_TILE, N, d, pitch);
-        load_rows(sg, G, head, i0, SIMT_TILE, N, d, pitch);
-        load_rows(sh, Hc, head, i0, SIMT_TILE, N, d, pitch);
+        load_rows(sq, Q, hq, qg.rs, i0, SIMT_TILE, M, d, pitch);
+        load_rows(stq, tQ, hq, qg.rs, i0, SIMT_TILE, M, d, pitch);
+        load_rows(sg, G, hq, qg.rs, i0, SIMT_TILE, M, d, pitch);
+        load_rows(sh, Hc, hq, qg.rs, i0, SIMT_TILE, M, d, pitch);
         __syncthreads();
-        const bool valid = i0 + lane < N;
-        const int i = min(i0 + lane, N - 1);
+        const bool valid = i0 + lane < M;
+        const int i = min(i0 + lane, M - 1);
         const float lse_i = lse[srow + i], mu_i = mu[srow + i], s1_i = sig1[srow + i], c_i = cvec[srow + i];
 #pragma unroll
         for (int r = 0; r < SIMT_RPW; ++r) {
@@ -432,7 +456,7 @@ simt_bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
         for (int k = 0; k < SIMT_MAXK; ++k) {
             const int c = lane + 32 * k;
             if (c < d) {
-                const size_t o = head + (size_t)j * d + c;
+                const size_t o = hk + (size_t)j * kg.rs + c;
                 from_f32(dK + o, alpha * aK[r][k]);
                 if (dtK) from_f32(dtK + o, alpha * aTK[r][k]);
                 from_f32(dV + o, aV[r][k]);

@@ -99,6 +99,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
         : "memory");
 }
 
+// The same for a 4-D tensor map (element, row, head, batch): tensors whose heads and batches have strides of
+// their own, e.g. a (B, rows, H, d) slice of a fused projection read in place.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
 // ---------------------------------------------------------------- tensor memory
 // Allocates `ncols` (power of two, 32..512) TMEM columns; the base address is written to *dst_smem.
 // Must be executed by one full warp.

@@ -41,29 +41,53 @@ struct Profiler {
 static Profiler g_prof;
 
 struct Shape {
-    int B, H, N, d, dp;
+    int B, H, N, M, d, dp;   // N keys, M queries per head
     long long BH;
     float alpha;
     bool fp32, simt;
+    Geom q, k;               // query side (M rows) and key side (N rows)
+    bool plain;              // self-attention on packed (B, H, N, d) tensors
 };
+
+// Strides of one side: all zero selects the packed (B, H, rows, d) layout.
+static int side_geometry(const int64_t st[3], int rows, int H, int d, Geom* g) {
+    g->rows = rows;
+    if (st[0] == 0 && st[1] == 0 && st[2] == 0) {
+        g->rs = d; g->hs = (long long)rows * d; g->bs = (long long)H * rows * d;
+        return TVM_ATTN_OK;
+    }
+    // rows must not overlap inside themselves and every row must start on a 16-byte boundary (TMA, vector loads)
+    if (st[0] < d || st[1] <= 0 || st[2] <= 0 || st[0] % 8 || st[1] % 8 || st[2] % 8) return TVM_ATTN_INVALID_ARG;
+    if (st[0] > (1LL << 36) || st[1] > (1LL << 36) || st[2] > (1LL << 36)) return TVM_ATTN_UNSUPPORTED;  // TMA strides < 2^40 bytes
+    g->rs = st[0]; g->hs = st[1]; g->bs = st[2];
+    return TVM_ATTN_OK;
+}
 
 static int check_params(const tvm_attn_params* p, Shape* s) {
     if (!p) return TVM_ATTN_INVALID_ARG;
-    if (p->B <= 0 || p->H <= 0 || p->N <= 0 || p->d <= 0) return TVM_ATTN_INVALID_ARG;
+    if (p->B <= 0 || p->H <= 0 || p->N <= 0 || p->d <= 0 || p->M < 0) return TVM_ATTN_INVALID_ARG;
     if (p->dtype != TVM_ATTN_BF16 && p->dtype != TVM_ATTN_FP32) return TVM_ATTN_INVALID_ARG;
     if (p->flags & ~TVM_ATTN_FLAG_CUDA_CORES) return TVM_ATTN_INVALID_ARG;
     if (!(p->scale >= 0.0f) || !std::isfinite(p->scale)) return TVM_ATTN_INVALID_ARG;
     if (p->d > 128 || p->d % 8 != 0) return TVM_ATTN_UNSUPPORTED;
     s->B = p->B; s->H = p->H; s->N = p->N; s->d = p->d;
+    s->M = p->M > 0 ? p->M : p->N;
+    int rg = side_geometry(p->q_strides, s->M, p->H, p->d, &s->q);
+    if (rg != TVM_ATTN_OK) return rg;
+    rg = side_geometry(p->k_strides, s->N, p->H, p->d, &s->k);
+    if (rg != TVM_ATTN_OK) return rg;
+    s->plain = s->M == s->N && s->q.rs == s->d && s->k.rs == s->d && s->q.hs == (long long)s->N * s->d && s->k.hs == s->q.hs &&
+               s->q.bs == (long long)s->H * s->N * s->d && s->k.bs == s->q.bs;
     s->dp = (p->d + 15) / 16 * 16;
     s->BH = (long long)p->B * p->H;
     s->alpha = p->scale == 0.0f ? 1.0f / std::sqrt((float)p->d) : p->scale;
     s->fp32 = p->dtype == TVM_ATTN_FP32;
     s->simt = s->fp32 || (p->flags & TVM_ATTN_FLAG_CUDA_CORES);
     // every kernel flattens (head, row tile) into blockIdx.x
-    const long long tiles16 = (p->N + 15LL) / 16;
+    const long long longer = s->M > s->N ? s->M : s->N;
+    const long long tiles16 = (longer + 15LL) / 16;
     if (s->BH * tiles16 > 2147483647LL) return TVM_ATTN_UNSUPPORTED;
-    if (s->BH > 2147483647LL / p->N) return TVM_ATTN_UNSUPPORTED;  // B*H*N rows indexable as int
+    if (s->BH > 2147483647LL / longer) return TVM_ATTN_UNSUPPORTED;  // B*H*rows indexable as int
     return TVM_ATTN_OK;
 }
 
@@ -79,20 +103,24 @@ static int simt_fwd(const Shape& s, const void* Q, const void* K, const void* V,
     const size_t smem = simt_smem_bytes(s.d, 2);
     cudaError_t e = cudaFuncSetAttribute(simt_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
-    const unsigned grid = (unsigned)(s.BH * ((s.N + SIMT_ROWS - 1) / SIMT_ROWS));
+    const unsigned grid = (unsigned)(s.BH * ((s.M + SIMT_ROWS - 1) / SIMT_ROWS));
     g_prof.before(st);
     simt_fwd_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
-                                                         (const T*)tK, (const T*)tV, (T*)O, (T*)tO, lse, mu, s.N, s.d,
-                                                         s.alpha);
+                                                         (const T*)tK, (const T*)tV, (T*)O, (T*)tO, lse, mu, s.q, s.k, s.H,
+                                                         s.d, s.alpha);
     g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
 }
 
+static bool q_packed(const Shape& s) {
+    return s.q.rs == s.d && s.q.hs == (long long)s.M * s.d && s.q.bs == (long long)s.H * s.M * s.d;
+}
+
 template <typename T>
 static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const void* O, const void* tO, const float* lse,
                           float* sig1, float* cvec, float* lse2, cudaStream_t st) {
-    const long long rows = s.BH * s.N;
+    const long long rows = s.BH * s.M;
     const int cpr = s.d * (int)sizeof(T) / 16;  // 16-byte chunks per row (d % 8 == 0)
     int gs = 1;
     while (gs < cpr) gs <<= 1;
@@ -101,7 +129,7 @@ static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const v
     const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
     g_prof.before(st);
     bwd_rowsums_kernel<T><<<grid, ROWSUM_THREADS, 0, st>>>((const T*)G, (const T*)Hc, (const T*)O, (const T*)tO, lse, sig1,
-                                                           cvec, lse2, rows, s.d, cpr, gs);
+                                                           cvec, lse2, rows, s.q, q_packed(s) ? 0 : s.H, s.d, cpr, gs);
     g_prof.after(st);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
@@ -116,15 +144,16 @@ static int simt_bwd(const Shape& s, const void* Q, const void* K, const void* V,
     if (cudaFuncSetAttribute(simt_bwd_dq_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
         cudaFuncSetAttribute(simt_bwd_dkv_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TVM_ATTN_CUDA_ERROR;
-    const unsigned grid = (unsigned)(s.BH * ((s.N + SIMT_ROWS - 1) / SIMT_ROWS));
-    simt_bwd_dq_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
-                                                            (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc, lse,
-                                                            mu, sig1, cvec, (T*)dQ, (T*)dtQ, s.N, s.d, s.alpha);
+    const unsigned grid_q = (unsigned)(s.BH * ((s.M + SIMT_ROWS - 1) / SIMT_ROWS));
+    const unsigned grid_k = (unsigned)(s.BH * ((s.N + SIMT_ROWS - 1) / SIMT_ROWS));
+    simt_bwd_dq_kernel<T><<<grid_q, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
+                                                              (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc, lse,
+                                                              mu, sig1, cvec, (T*)dQ, (T*)dtQ, s.q, s.k, s.H, s.d, s.alpha);
     g_prof.after(st);
-    simt_bwd_dkv_kernel<T><<<grid, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
-                                                             (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc,
-                                                             lse, mu, sig1, cvec, (T*)dK, (T*)dV, (T*)dtK, (T*)dtV,
-                                                             s.N, s.d, s.alpha);
+    simt_bwd_dkv_kernel<T><<<grid_k, SIMT_THREADS, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)tQ,
+                                                               (const T*)tK, (const T*)tV, (const T*)G, (const T*)Hc,
+                                                               lse, mu, sig1, cvec, (T*)dK, (T*)dV, (T*)dtK, (T*)dtV,
+                                                               s.q, s.k, s.H, s.d, s.alpha);
     g_prof.after(st);
     g_launches += 2;
     return cuda_status(cudaGetLastError());
@@ -149,9 +178,23 @@ static encode_tiled_fn get_encode_fn() {
     return fn;
 }
 
-// (B,H,N,d) bf16 viewed as a 3-D tensor (d, N, B*H); a box is 64 columns x `rows` rows of one head with
-// the 128-byte swizzle; columns or rows beyond the tensor read as zero.
-static int make_tmap(CUtensorMap* m, const void* ptr, const Shape& s, int rows) {
+// A bf16 tensor of one side viewed as a 4-D tensor (d, rows, H, B) with that side's strides; a box is 64 columns x
+// `rows` rows of one head with the 128-byte swizzle; columns or rows beyond the tensor read as zero.
+static int make_tmap(CUtensorMap* m, const void* ptr, const Shape& s, const Geom& g, int rows) {
+    encode_tiled_fn fn = get_encode_fn();
+    if (!fn) return TVM_ATTN_CUDA_ERROR;
+    cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)g.rows, (cuuint64_t)s.H, (cuuint64_t)s.B};
+    cuuint64_t strides[3] = {(cuuint64_t)g.rs * 2, (cuuint64_t)g.hs * 2, (cuuint64_t)g.bs * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TVM_ATTN_OK : TVM_ATTN_CUDA_ERROR;
+}
+
+// Packed (B,H,N,d) bf16 viewed as a 3-D tensor (d, N, B*H): the kernels for head dims above 80.
+static int make_tmap3(CUtensorMap* m, const void* ptr, const Shape& s, int rows) {
     encode_tiled_fn fn = get_encode_fn();
     if (!fn) return TVM_ATTN_CUDA_ERROR;
     cuuint64_t dims[3] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.BH};
@@ -184,9 +227,9 @@ static int launch_tc(const Shape& s, const void* const own[4], const void* const
     CUtensorMap mo[4], ms[4];
     for (int t = 0; t < 4; ++t) {
         const void* po = own[t < C::NOWN ? t : 0];
-        int rc = make_tmap(&mo[t], po, s, TC_OWN_ROWS);
+        int rc = make_tmap3(&mo[t], po, s, TC_OWN_ROWS);
         if (rc != TVM_ATTN_OK) return rc;
-        rc = make_tmap(&ms[t], strm[t], s, C::BC);
+        rc = make_tmap3(&ms[t], strm[t], s, C::BC);
         if (rc != TVM_ATTN_OK) return rc;
     }
     auto kern = dual_attn_kernel<MODE, NA>;
@@ -212,7 +255,7 @@ static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams
     using C = FwdCfg<DP>;
     CUtensorMap m[4];
     for (int t = 0; t < 4; ++t) {
-        const int rc = make_tmap(&m[t], strm[t], s, FWD_BC);
+        const int rc = make_tmap(&m[t], strm[t], s, s.k, FWD_BC);
         if (rc != TVM_ATTN_OK) return rc;
     }
     auto kern = jvp_fwd_kernel<DP>;
@@ -220,7 +263,7 @@ static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams
         return TVM_ATTN_CUDA_ERROR;
     // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
     // items go round-robin over them
-    const long long items = s.BH * ((s.N + FWD_ROWS - 1) / FWD_ROWS);
+    const long long items = s.BH * ((s.M + FWD_ROWS - 1) / FWD_ROWS);
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return TVM_ATTN_CUDA_ERROR;
@@ -237,15 +280,18 @@ template <int MODE, int DP>
 static int launch_bwd_pass(const Shape& s, const void* const own[4], const void* const strm[4], BwdParams prm, cudaStream_t st) {
     using C = BwdCfg<MODE, DP>;
     CUtensorMap ms[4], mo[2];
+    // DV, DK: keys own, queries stream; DQ: queries own, keys stream
+    prm.o = MODE == BWD_DQ ? s.q : s.k;
+    prm.s = MODE == BWD_DQ ? s.k : s.q;
     for (int t = 0; t < 4; ++t) {
         // an absent cotangent (null) is never loaded: its map is built on a present tensor and stays unused
-        const int rc = make_tmap(&ms[t], strm[t] ? strm[t] : strm[t ^ 1], s, C::BC);
+        const int rc = make_tmap(&ms[t], strm[t] ? strm[t] : strm[t ^ 1], s, prm.s, C::BC);
         if (rc != TVM_ATTN_OK) return rc;
         prm.strm[t] = static_cast<const __nv_bfloat16*>(strm[t]);
         prm.own[t] = static_cast<const __nv_bfloat16*>(own[t]);
     }
     for (int t = 0; t < 2; ++t) {
-        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? C::XS0 + t : t], s, BWD_ROWS);  // never a cotangent
+        const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? C::XS0 + t : t], s, prm.o, BWD_ROWS);  // never a cotangent
         if (rc != TVM_ATTN_OK) return rc;
     }
     auto kern = jvp_bwd_kernel<MODE, DP>;
@@ -253,7 +299,7 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
         return TVM_ATTN_CUDA_ERROR;
     // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
     // items go round-robin over them
-    const long long items = s.BH * ((s.N + BWD_ROWS - 1) / BWD_ROWS);
+    const long long items = s.BH * ((prm.o.rows + BWD_ROWS - 1) / BWD_ROWS);
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return TVM_ATTN_CUDA_ERROR;
@@ -364,10 +410,12 @@ static int rms_fwd(const Shape& s, float eps, const void* Q, const void* tQ, con
     int cpr, gs;
     const int rc = rms_geometry(s, &cpr, &gs);
     if (rc != TVM_ATTN_OK) return rc;
-    const long long rows = s.BH * s.N, rows_per_block = (long long)(RMS_THREADS / 32) * (32 / gs);
-    const RmsFwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (T*)Qn, (T*)tQn}, k{(const T*)K, (const T*)tK, gK, (T*)Kn, (T*)tKn};
+    const long long rows_q = s.BH * s.M, rows_k = s.BH * s.N, rows_per_block = (long long)(RMS_THREADS / 32) * (32 / gs);
+    const RmsFwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (T*)Qn, (T*)tQn, s.q, rows_q};
+    const RmsFwdSide<T> k{(const T*)K, (const T*)tK, gK, (T*)Kn, (T*)tKn, s.k, rows_k};
+    const long long rows = rows_q > rows_k ? rows_q : rows_k;
     const dim3 grid((unsigned)((rows + rows_per_block - 1) / rows_per_block), 2);
-    qk_rmsnorm_jvp_fwd_kernel<T><<<grid, RMS_THREADS, 0, st>>>(q, k, rows, s.d, cpr, gs, eps);
+    qk_rmsnorm_jvp_fwd_kernel<T><<<grid, RMS_THREADS, 0, st>>>(q, k, s.H, s.d, cpr, gs, eps);
     g_launches += 1;
     return cuda_status(cudaGetLastError());
 }
@@ -379,12 +427,11 @@ static int rms_bwd(const Shape& s, float eps, const void* Q, const void* tQ, con
     int cpr, gs;
     const int rc = rms_geometry(s, &cpr, &gs);
     if (rc != TVM_ATTN_OK) return rc;
-    const long long rows = s.BH * s.N;
     float* pq = partial;
     float* pk = partial + (size_t)RMS_BWD_BLOCKS * s.d;
-    const RmsBwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (const T*)dQn, (const T*)dtQn, (T*)dQ, (T*)dtQ, pq};
-    const RmsBwdSide<T> k{(const T*)K, (const T*)tK, gK, (const T*)dKn, (const T*)dtKn, (T*)dK, (T*)dtK, pk};
-    qk_rmsnorm_jvp_bwd_kernel<T><<<dim3(RMS_BWD_BLOCKS, 2), RMS_THREADS, 0, st>>>(q, k, rows, s.d, cpr, gs, eps);
+    const RmsBwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (const T*)dQn, (const T*)dtQn, (T*)dQ, (T*)dtQ, pq, s.q, s.BH * s.M};
+    const RmsBwdSide<T> k{(const T*)K, (const T*)tK, gK, (const T*)dKn, (const T*)dtKn, (T*)dK, (T*)dtK, pk, s.k, s.BH * s.N};
+    qk_rmsnorm_jvp_bwd_kernel<T><<<dim3(RMS_BWD_BLOCKS, 2), RMS_THREADS, 0, st>>>(q, k, s.H, s.d, cpr, gs, eps);
     qk_rmsnorm_dg_reduce_kernel<<<2, 128, 0, st>>>(pq, pk, dgQ, dgK, RMS_BWD_BLOCKS, s.d);
     g_launches += 2;
     return cuda_status(cudaGetLastError());
@@ -402,7 +449,7 @@ size_t tvm_attn_jvp_workspace_bytes(const tvm_attn_params* p, int is_bwd) {
     Shape s;
     if (check_params(p, &s) != TVM_ATTN_OK) return 0;
     if (!is_bwd) return 0;
-    return (size_t)3 * sizeof(float) * (size_t)s.BH * (size_t)s.N;
+    return (size_t)3 * sizeof(float) * (size_t)s.BH * (size_t)s.M;   // per query row
 }
 
 int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, const void* V, const void* tQ,
@@ -428,7 +475,7 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
     const void* strm[4] = {K, tK, V, tV};
     if (s.dp <= 80) {
         FwdParams f;
-        f.N = s.N; f.d = s.d; f.BH = (int)s.BH;
+        f.d = s.d; f.BH = (int)s.BH; f.H = s.H; f.q = s.q; f.k = s.k;
         f.alpha = s.alpha; f.c2 = s.alpha * 1.4426950408889634f;
         f.Q = static_cast<const __nv_bfloat16*>(Q); f.tQ = static_cast<const __nv_bfloat16*>(tQ);
         f.K = static_cast<const __nv_bfloat16*>(K); f.tK = static_cast<const __nv_bfloat16*>(tK);
@@ -443,6 +490,7 @@ int tvm_attn_jvp_fwd(const tvm_attn_params* p, const void* Q, const void* K, con
             default: return launch_fwd<80>(s, strm, f, st);
         }
     }
+    if (!s.plain) return TVM_ATTN_UNSUPPORTED;  // head dims above 80: self-attention on packed tensors only
     TcParams prm = base_params(s, status);
     prm.out0 = O; prm.out1 = tO; prm.lse_out = lse; prm.mu_out = mu;
     const void* own[4] = {Q, tQ, Q, tQ};
@@ -467,19 +515,25 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
         if (x && !aligned16(x)) return TVM_ATTN_INVALID_ARG;
     if (dtO && (!dtQ || !dtK || !dtV)) return TVM_ATTN_INVALID_ARG;
     const int absent = (dtO ? 0 : ABSENT_HC) | (dO ? 0 : ABSENT_G);
-    if (absent && !s.simt && s.dp > 80) return TVM_ATTN_UNSUPPORTED;  // head dims above 80 need both cotangents
-    const size_t rows = (size_t)s.BH * (size_t)s.N;
+    if ((absent || !s.plain) && !s.simt && s.dp > 80) return TVM_ATTN_UNSUPPORTED;  // head dims above 80: both cotangents, packed self-attention
+    const size_t rows = (size_t)s.BH * (size_t)s.M;   // query rows: what the workspace and the statistics are sized by
     if (workspace_bytes < 3 * sizeof(float) * rows) return TVM_ATTN_WORKSPACE_TOO_SMALL;
     float* sig1 = static_cast<float*>(workspace);
     float* cvec = sig1 + rows;
     float* lse2 = cvec + rows;  // lse * log2(e)
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     g_prof.begin_call();
-    if (!dtO) {  // the tangent gradients of a call without dtO are zero: written here, by no kernel
-        const size_t bytes = rows * (size_t)s.d * (s.fp32 ? 4 : 2);
+    if (!dtO) {  // the tangent gradients of a call without dtO are zero: written here, by none of the passes
         void* zero_out[] = {dtQ, dtK, dtV};
-        for (void* z : zero_out)
-            if (z && cudaMemsetAsync(z, 0, bytes, st) != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+        const int esz = s.fp32 ? 4 : 2, cpr = s.d * esz / 16;
+        for (int i = 0; i < 3; ++i) {
+            if (!zero_out[i]) continue;
+            const Geom& g = i == 0 ? s.q : s.k;
+            const long long zr = s.BH * g.rows, n = zr * cpr;
+            zero_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(static_cast<uint4*>(zero_out[i]), g, s.H, zr, cpr, 16 / esz);
+            g_launches += 1;
+            if (cudaGetLastError() != cudaSuccess) return TVM_ATTN_CUDA_ERROR;
+        }
     }
     if (s.simt) {
         if (s.fp32) {
@@ -500,7 +554,7 @@ int tvm_attn_jvp_bwd(const tvm_attn_params* p, const void* Q, const void* K, con
     if (s.dp <= 80) {
         BwdParams b;
         std::memset(&b, 0, sizeof b);
-        b.N = s.N; b.d = s.d; b.BH = (int)s.BH;
+        b.d = s.d; b.BH = (int)s.BH; b.H = s.H;
         b.alpha = s.alpha; b.c2 = s.alpha * 1.4426950408889634f;
         b.lse2 = lse2; b.mu = mu; b.sig1 = sig1; b.cvec = cvec; b.status = status; b.absent = absent;
         {   // dtV = P^T Hc, dV = P^T G + (P*Nn)^T Hc : owner keys (K, tK); stream queries (Q, tQ | Hc, G)
@@ -560,7 +614,7 @@ int tvm_attn_jvp_bwd_noalloc(const tvm_attn_params* p, const void* Q, const void
     Shape s;
     const int rc = check_params(p, &s);
     if (rc != TVM_ATTN_OK) return rc;
-    if (s.BH * (long long)s.N > (long long)TVM_ATTN_NOALLOC_MAX_ROWS) return TVM_ATTN_TOO_LARGE;
+    if (s.BH * (long long)s.M > (long long)TVM_ATTN_NOALLOC_MAX_ROWS) return TVM_ATTN_TOO_LARGE;
     float* scratch = nullptr;
     const int rs = noalloc_scratch_address(&scratch);
     if (rs != TVM_ATTN_OK) return rs;
