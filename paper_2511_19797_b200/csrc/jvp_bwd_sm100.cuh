@@ -145,7 +145,10 @@ struct BwdCfg {
 };
 
 // Element-wise warps of the backward passes: `w` in 0..15.
-template <int MODE, int DP>
+// HZ: the cotangent Hc = dtO is absent (the "detach JVP" setting), known at compile time: everything that only
+// feeds the tangent path is left out -- Sd, Nn, D, W and their MMAs -- and what remains is the standard attention
+// backward: P from S, dA = P (G V^T - rowsum(G O)), dV = P^T G, dK = alpha dA^T Q, dQ = alpha dA K.
+template <int MODE, int DP, bool HZ>
 __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tmem_base, uint32_t bar0,
                                                 volatile int* abort_flag, const float* stats, int w, int lane, int items,
                                                 int row_tiles, int T) {
@@ -245,14 +248,25 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 const float* stt = st + 16 * sub;
                 uint32_t s1[16], s2[16];
                 ptx::tmem_ld16(sb, s1);
-                ptx::tmem_ld16(sb + BC, s2);
+                if (!HZ) ptx::tmem_ld16(sb + BC, s2);
                 ptx::tmem_wait_ld();
                 uint32_t pa0[8], pa1[8];
 #pragma unroll
                 for (int c4 = 0; c4 < 16; c4 += 4) {
                     const float4 l4 = *reinterpret_cast<const float4*>(stt + c4);
+                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+                    if (HZ) {  // P only
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
+                            float x0, x1;
+                            ptx::unpack2(x2, x0, x1);
+                            pa0[(c4 + e) >> 1] = ptx::pack_bf16(ptx::ex2(x0), ptx::ex2(x1));
+                        }
+                        continue;
+                    }
                     const float4 m4 = *reinterpret_cast<const float4*>(stt + 64 + c4);
-                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
+                    const float mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
                     for (int e = 0; e < 4; e += 2) {  // P = 2^(c2 s - lse2), P Nn with Nn = alpha ts - mu: two columns per instruction
                         const uint64_t x2 = ptx::fma2(ptx::pack2u(s1[c4 + e], s1[c4 + e + 1]), c2c2, ptx::pack2(-lv[e], -lv[e + 1]));
@@ -269,7 +283,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 }
                 // operand of a k-step (16 stream rows) sits at the slice's columns of the accumulator it replaces
                 ptx::tmem_st8(sb, pa0);
-                ptx::tmem_st8(sb + BC, pa1);
+                if (!HZ) ptx::tmem_st8(sb + BC, pa1);
               }
             } else {
                 // ---- phase A: P, Nn, -P Sigma1, -P c from (S, Sd), two columns per register pair; then that half of the
@@ -279,7 +293,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 {
                     uint32_t s1[16], s2[16];
                     ptx::tmem_ld16(sbase, s1);
-                    ptx::tmem_ld16(sbase + BC, s2);
+                    if (!HZ) ptx::tmem_ld16(sbase + BC, s2);
                     ptx::tmem_wait_ld();
                     ptx::tc_fence_before_sync();
                     __syncwarp();
@@ -311,8 +325,10 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                             float x0, x1;
                             ptx::unpack2(x2, x0, x1);
                             P2[k] = ptx::pack2(ptx::ex2(x0), ptx::ex2(x1));
-                            Nn2[k] = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
-                            nPs2[k] = ptx::mul2(P2[k], ptx::pack2(-gv[e], -gv[e + 1]));
+                            if (!HZ) {
+                                Nn2[k] = ptx::fma2(ptx::pack2u(s2[c4 + e], s2[c4 + e + 1]), aa, ptx::pack2(-mv[e], -mv[e + 1]));
+                                nPs2[k] = ptx::mul2(P2[k], ptx::pack2(-gv[e], -gv[e + 1]));
+                            }
                             nPc2[k] = ptx::mul2(P2[k], ptx::pack2(-cv[e], -cv[e + 1]));
                         }
                     }
@@ -321,22 +337,27 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 if (!ptx::mbar_wait_warp(bar(C::B_SFULL + 1), g & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
                 uint32_t s3[16], s4[16];
-                ptx::tmem_ld16(sbase + 2 * BC, s3);
+                if (!HZ) ptx::tmem_ld16(sbase + 2 * BC, s3);
                 ptx::tmem_ld16(sbase + 3 * BC, s4);
                 ptx::tmem_wait_ld();
                 uint32_t pa0[8], pa1[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const uint64_t w2 = ptx::fma2(P2[k], ptx::pack2u(s3[2 * k], s3[2 * k + 1]), nPs2[k]);
                     const uint64_t t2 = ptx::fma2(P2[k], ptx::pack2u(s4[2 * k], s4[2 * k + 1]), nPc2[k]);
-                    const uint64_t d2 = ptx::fma2(w2, Nn2[k], t2);
-                    float w0, w1, d0, d1;
-                    ptx::unpack2(w2, w0, w1);
-                    ptx::unpack2(d2, d0, d1);
-                    pa0[k] = ptx::pack_bf16(w0, w1);
+                    float d0, d1;
+                    if (HZ) {  // dA = P (X - c): no W
+                        ptx::unpack2(t2, d0, d1);
+                    } else {
+                        const uint64_t w2 = ptx::fma2(P2[k], ptx::pack2u(s3[2 * k], s3[2 * k + 1]), nPs2[k]);
+                        const uint64_t d2 = ptx::fma2(w2, Nn2[k], t2);
+                        float w0, w1;
+                        ptx::unpack2(w2, w0, w1);
+                        ptx::unpack2(d2, d0, d1);
+                        pa0[k] = ptx::pack_bf16(w0, w1);
+                    }
                     pa1[k] = ptx::pack_bf16(d0, d1);
                 }
-                ptx::tmem_st8(sbase + 2 * BC, pa0);
+                if (!HZ) ptx::tmem_st8(sbase + 2 * BC, pa0);
                 ptx::tmem_st8(sbase + 3 * BC, pa1);
             }
             ptx::tmem_wait_st();
@@ -388,7 +409,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     }
 }
 
-template <int MODE, int DP>
+template <int MODE, int DP, bool HZ>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant__ CUtensorMap tm_s1,
                const __grid_constant__ CUtensorMap tm_s2, const __grid_constant__ CUtensorMap tm_s3,
@@ -468,7 +489,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             ptx::fence_proxy_async_smem();
         }
     }
-    if (MODE == BWD_DK && p.absent) {
+    if (MODE == BWD_DK && p.absent && !HZ) {
         // DK reads both cotangent tiles of an E stage in one N = 128 MMA: the never-loaded one must read as zero
         const int t = (p.absent & ABSENT_HC) ? 0 : 1;
         for (int i = threadIdx.x; i < SE * BC * 8; i += BWD_THREADS) {  // the 64-column atoms, 16 bytes at a time
@@ -754,14 +775,16 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
 #pragma unroll
             for (int kk = 0; kk < KS; ++kk)  // S = X0 Y0^T
                 ptx::mma_ts_elect(dS, ax0 + 8 * kk, desc64(e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL), idesc_s, kk > 0 ? 1u : 0u);
+            if (!HZ) {
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk)  // Sd = X1 Y0^T
-                ptx::mma_ts_elect(dT, ax1 + 8 * kk, desc64(e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL), idesc_s, kk > 0 ? 1u : 0u);
+                for (int kk = 0; kk < KS; ++kk)  // Sd = X1 Y0^T
+                    ptx::mma_ts_elect(dT, ax1 + 8 * kk, desc64(e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk)  // Sd += X0 Y1^T
-                ptx::mma_ts_elect(dT, ax0 + 8 * kk,
-                                  kk < 4 ? desc64(ptx::desc_lo(y1, 16) + 2u * kk, HI_SW128) : desc64(ptx::desc_lo(y1t, 2 * BC * 16), HI_TAIL),
-                                  idesc_s, 1u);
+                for (int kk = 0; kk < KS; ++kk)  // Sd += X0 Y1^T
+                    ptx::mma_ts_elect(dT, ax0 + 8 * kk,
+                                      kk < 4 ? desc64(ptx::desc_lo(y1, 16) + 2u * kk, HI_SW128) : desc64(ptx::desc_lo(y1t, 2 * BC * 16), HI_TAIL),
+                                      idesc_s, 1u);
+            }
             ptx::mma_commit_elect(bar(C::B_SFULL + b));
             ptx::mma_commit_elect(bar(C::B_EEMPTY + g % SE));
             return true;
@@ -780,7 +803,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const uint64_t b0 = desc64(l_nlo(l_stage(g), 0, 0), HI_SW128);
             const uint64_t b1 = desc64(l_nlo(l_stage(g), 1, 0), HI_SW128);
             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
-            const bool hasH = !(p.absent & ABSENT_HC), hasG = !(p.absent & ABSENT_G);  // B0 = Hc, B1 = G
+            const bool hasH = !HZ && !(p.absent & ABSENT_HC), hasG = !(p.absent & ABSENT_G);  // B0 = Hc, B1 = G
 #pragma unroll
             for (int u = 0; u < BC / 16; ++u) {
                 const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
@@ -841,14 +864,16 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                     const uint32_t el = ptx::elect_one();
                     const uint32_t st = l_stage(g);
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) {
+                    for (int kk = 0; kk < KS; ++kk) {  // HZ: S = X0 Y0^T alone
                         const uint32_t ahi = kk < 4 ? HI_SW128 : HI_TAIL;
-                        if (kk == 0) ptx::mma_ss_p<0>(el, dS, own_klo(own_base, kk), ahi, l_klo(st, kk), HI_SW128, idesc_s2);
-                        else ptx::mma_ss_p<1>(el, dS, own_klo(own_base, kk), ahi, l_klo(st, kk), HI_SW128, idesc_s2);
+                        if (kk == 0) ptx::mma_ss_p<0>(el, dS, own_klo(own_base, kk), ahi, l_klo(st, kk), HI_SW128, HZ ? idesc_s : idesc_s2);
+                        else ptx::mma_ss_p<1>(el, dS, own_klo(own_base, kk), ahi, l_klo(st, kk), HI_SW128, HZ ? idesc_s : idesc_s2);
                     }
+                    if (!HZ) {
 #pragma unroll
-                    for (int kk = 0; kk < KS; ++kk)
-                        ptx::mma_ss_p<1>(el, dT, own_klo(own_base + C::OWN_BYTES, kk), kk < 4 ? HI_SW128 : HI_TAIL, l_klo(st, kk), HI_SW128, idesc_s);
+                        for (int kk = 0; kk < KS; ++kk)
+                            ptx::mma_ss_p<1>(el, dT, own_klo(own_base + C::OWN_BYTES, kk), kk < 4 ? HI_SW128 : HI_TAIL, l_klo(st, kk), HI_SW128, idesc_s);
+                    }
                     ptx::mma_commit_p(el, bar(C::B_SFULL + 0));
                     if (last) ptx::mma_commit_p(el, bar(C::B_OWNFREE));
                 };
@@ -856,6 +881,21 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                 auto issue_second_pair = [&](int g) {
                     const uint32_t el = ptx::elect_one();
                     const uint32_t st = e_stage(g);
+                    if (HZ) {
+                        // X = G V^T alone.  DK: X2 Y3^T with X2 = V in tensor memory and Y3 = G the second tensor of the E
+                        // stage; DQ: X3 Y2^T with X3 = G in tensor memory and Y2 = V the first tensor of the stage.
+                        const uint32_t ya = MODE == BWD_DK ? st + BC * 128 : st, yt = st + 2 * BC * 128 + (MODE == BWD_DK ? BC * 16 : 0);
+                        const uint32_t ax = MODE == BWD_DK ? ax0 : ax1;
+#pragma unroll
+                        for (int kk = 0; kk < KS; ++kk) {
+                            const uint32_t lo = kk < 4 ? ptx::desc_lo(ya, 16) + 2u * kk : ptx::desc_lo(yt, 2 * BC * 16);
+                            if (kk == 0) ptx::mma_ts_p<0>(el, dX, ax + 8 * kk, lo, kk < 4 ? HI_SW128 : HI_TAIL, idesc_s);
+                            else ptx::mma_ts_p<1>(el, dX, ax + 8 * kk, lo, kk < 4 ? HI_SW128 : HI_TAIL, idesc_s);
+                        }
+                        ptx::mma_commit_p(el, bar(C::B_SFULL + 1));
+                        ptx::mma_commit_p(el, bar(C::B_EEMPTY + g % SE));
+                        return;
+                    }
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
                         if (kk == 0) ptx::mma_ts_p<0>(el, dD, ax0 + 8 * kk, e_klo(st, kk), kk < 4 ? HI_SW128 : HI_TAIL, idesc_s2);
@@ -907,7 +947,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                         {
                             const uint32_t el = ptx::elect_one();
                             const uint32_t b0 = l_nlo(l_stage(g), 0, 0), b1 = l_nlo(l_stage(g), 1, 0);  // MN-major B
-                            const bool hasW = !(p.absent & ABSENT_HC);
+                            const bool hasW = !HZ && !(p.absent & ABSENT_HC);
                             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
 #pragma unroll
                             for (int u = 0; u < BC / 16; ++u) {
@@ -931,7 +971,7 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             }
         }
     } else {
-        bwd_elementwise<MODE, DP>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, items, row_tiles, T);
+        bwd_elementwise<MODE, DP, HZ>(p, tmem_base, bar0, abort_flag, stats, warp - 4, lane, items, row_tiles, T);
     }
 
     // ---------------------------------------------------------------------- teardown

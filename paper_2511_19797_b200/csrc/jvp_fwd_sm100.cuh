@@ -92,7 +92,8 @@ struct FwdCfg {
     static constexpr int B_QREADY = B_FINAL + 1;
     static constexpr int B_XMAX = B_QREADY + 1;   // per quadrant: slice maxima exchanged
     static constexpr int B_XSLOW = B_XMAX + 4;    // per quadrant: slow-path / epilogue exchange
-    static constexpr int NBARS = B_XSLOW + 4;
+    static constexpr int B_DRAIN = B_XSLOW + 4;   // + issuer: used once, while winding down after a time-out
+    static constexpr int NBARS = B_DRAIN + 2;
     static_assert(NBARS <= 48, "barrier table too small");
     static constexpr int XMAX_FLOATS = 2 * 128 * 4;   // [parity][row][slice]
     static constexpr int XSLOW_FLOATS = 2 * 128 * 4 * 2;  // [exchange parity][row][slice][2]
@@ -429,6 +430,8 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         ptx::mbar_init(bar(C::B_FINAL), 1);
         ptx::mbar_init(bar(C::B_QREADY), 16);
         for (int q = 0; q < 4; ++q) { ptx::mbar_init(bar(C::B_XMAX + q), 4); ptx::mbar_init(bar(C::B_XSLOW + q), 4); }
+        ptx::mbar_init(bar(C::B_DRAIN), 1);
+        ptx::mbar_init(bar(C::B_DRAIN + 1), 1);
         ptx::fence_mbar_init();
     }
     if (NA == 2) {
@@ -538,10 +541,19 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         if (NA == 2) {
             ptx::cp_async_wait<0>();  // nothing of ours stays in flight
-            if (ok && pend_s >= 0) {
+            if (pend_s >= 0) {       // (also after a time-out: the drain below waits for these barriers)
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(b_full + pend_s));
+            }
+        }
+        if (!ok) {
+            // Winding down after a time-out: the TMA loads this warp started write into this block's shared memory
+            // and must have landed before the block exits.  Stages below s carry the phase of this pass over the
+            // ring, the others the one before.
+            for (int k = 0; k < S; ++k) {
+                const bool cur = k < s;
+                ptx::mbar_wait_drain(bar(b_full + k), (cur ? ph : ph ^ 1) & 1, ptx::DRAIN_LIMIT_NS);
             }
         }
     } else if (warp == 1) {
@@ -626,6 +638,11 @@ jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     }
 
     // ---------------------------------------------------------------------- teardown
+    if ((warp == 1 || warp == 3) && *abort_flag) {
+        // after a time-out: the MMAs this warp queued must be done before the tensor memory is given back
+        ptx::mma_commit_elect(bar(C::B_DRAIN + (warp >> 1)));
+        ptx::mbar_wait_drain(bar(C::B_DRAIN + (warp >> 1)), 0, ptx::DRAIN_LIMIT_NS);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {

@@ -294,7 +294,10 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
         const int rc = make_tmap(&mo[t], own[C::NPAIR == 2 ? C::XS0 + t : t], s, prm.o, BWD_ROWS);  // never a cotangent
         if (rc != TVM_ATTN_OK) return rc;
     }
-    auto kern = jvp_bwd_kernel<MODE, DP>;
+    // dtO absent: the specialisation that leaves the tangent path out (only instantiated for the padded head dims
+    // 64 and 80 of the transformer shapes; other head dims run the general kernel, which skips what it can)
+    constexpr bool HAS_HZ = DP == 64 || DP == 80;
+    auto kern = (HAS_HZ && (prm.absent & ABSENT_HC)) ? jvp_bwd_kernel<MODE, DP, HAS_HZ> : jvp_bwd_kernel<MODE, DP, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
         return TVM_ATTN_CUDA_ERROR;
     // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
