@@ -18,4 +18,20 @@ struct Geom {
     }
 };
 
+#ifdef __CUDACC__
+// Sum of v over the `gs` consecutive lanes of a warp that share a row (lanes sub * gs .. sub * gs + gs - 1), returned
+// to all of them.  A power-of-two group is a butterfly; any other size (nine 16-byte chunks for d = 72) has its first
+// lane collect the others' values and broadcast the total, which keeps 27 of 32 lanes busy where rounding the group
+// up to 16 lanes would leave 14 idle.  Executed by the whole warp.
+__device__ __forceinline__ float lane_group_sum(float v, int gs, int lane) {
+    if ((gs & (gs - 1)) == 0) {
+        for (int off = gs >> 1; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        return v;
+    }
+    float acc = v;
+    for (int k = 1; k < gs; ++k) acc += __shfl_sync(0xffffffffu, v, lane + k);   // right on the group's first lane
+    return __shfl_sync(0xffffffffu, acc, lane - lane % gs);
+}
+#endif
+
 }  // namespace tvm_attn

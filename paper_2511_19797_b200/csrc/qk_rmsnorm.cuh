@@ -57,11 +57,6 @@ __device__ __forceinline__ void rms_load_scale(const float* g, float (&v)[N]) {
         v[i] = q.x; v[i + 1] = q.y; v[i + 2] = q.z; v[i + 3] = q.w;
     }
 }
-// Sum over the `gs` lanes (a power of two) that share a row.
-__device__ __forceinline__ float rms_group_sum(float v, int gs) {
-    for (int off = gs >> 1; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-    return v;
-}
 
 template <typename T>
 struct RmsFwdSide {
@@ -79,7 +74,7 @@ qk_rmsnorm_jvp_fwd_kernel(const RmsFwdSide<T> q, const RmsFwdSide<T> k, int H, i
     const int lane = threadIdx.x & 31, rpw = 32 / gs;
     const int sub = lane / gs, c = lane - sub * gs;
     const long long row = ((long long)blockIdx.x * (RMS_THREADS / 32) + (threadIdx.x >> 5)) * rpw + sub;
-    const bool act = row < a.rows && c < cpr;
+    const bool act = row < a.rows && c < cpr && sub < rpw;
     float x[V], t[V], g[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) x[i] = t[i] = g[i] = 0.f;
@@ -93,8 +88,8 @@ qk_rmsnorm_jvp_fwd_kernel(const RmsFwdSide<T> q, const RmsFwdSide<T> k, int H, i
     float ss = 0.f, s = 0.f;
 #pragma unroll
     for (int i = 0; i < V; ++i) { ss = fmaf(x[i], x[i], ss); s = fmaf(x[i], t[i], s); }
-    ss = rms_group_sum(ss, gs);
-    s = rms_group_sum(s, gs);
+    ss = lane_group_sum(ss, gs, lane);
+    s = lane_group_sum(s, gs, lane);
     const float inv = 1.0f / sqrtf(ss / (float)d + eps);
     const float m = s * inv * inv / (float)d;   // (u . tx) / (d r)
     if (act) {
@@ -127,7 +122,7 @@ struct RmsBwdSide {
 // block then adds them up in a fixed order and writes one partial row; a second kernel adds the partial rows, again
 // in a fixed order, so dg is bit-reproducible.
 template <typename T>
-__global__ void __launch_bounds__(RMS_THREADS)
+__global__ void __launch_bounds__(RMS_THREADS, 3)
 qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, int H, int d, int cpr, int gs, float eps) {
     constexpr int V = RmsVec<T>::N;
     __shared__ float part[(RMS_THREADS / 32) * 32 * V];   // [warp][row in warp][column]; d * rows-per-warp <= 32 * V
@@ -138,12 +133,12 @@ qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, int H, i
     float g[V], dg[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) g[i] = dg[i] = 0.f;
-    if (c < cpr) rms_load_scale<V>(a.g + c * V, g);
+    if (c < cpr && sub < rpw) rms_load_scale<V>(a.g + c * V, g);
     const float fd = (float)d;
     const long long rows = a.rows;
     for (long long base = (long long)blockIdx.x * rows_per_block; base < rows; base += (long long)gridDim.x * rows_per_block) {
         const long long row = base + (long long)warp * rpw + sub;
-        const bool act = row < rows && c < cpr;
+        const bool act = row < rows && c < cpr && sub < rpw;
         float x[V], t[V], gy[V], gt[V];
 #pragma unroll
         for (int i = 0; i < V; ++i) x[i] = t[i] = gy[i] = gt[i] = 0.f;
@@ -165,11 +160,11 @@ qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, int H, i
             bx = fmaf(bi, x[i], bx);
             bt = fmaf(bi, t[i], bt);
         }
-        ss = rms_group_sum(ss, gs);
-        s = rms_group_sum(s, gs);
-        ax = rms_group_sum(ax, gs);
-        bx = rms_group_sum(bx, gs);
-        bt = rms_group_sum(bt, gs);
+        ss = lane_group_sum(ss, gs, lane);
+        s = lane_group_sum(s, gs, lane);
+        ax = lane_group_sum(ax, gs, lane);
+        bx = lane_group_sum(bx, gs, lane);
+        bt = lane_group_sum(bt, gs, lane);
         const float inv = 1.0f / sqrtf(ss / fd + eps);
         const float inv2 = inv * inv, k3 = inv2 * inv / fd;
         const float au_d = ax * inv / fd, bu_d = bx * inv / fd;   // (a.u)/d, (b.u)/d
@@ -191,7 +186,7 @@ qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, int H, i
     }
     // ---- dg of the block, in a fixed order
     float* mine = part + (warp * rpw + sub) * d + c * V;
-    if (c < cpr) {
+    if (c < cpr && sub < rpw) {
 #pragma unroll
         for (int i = 0; i < V; ++i) mine[i] = dg[i];
     }
@@ -203,16 +198,25 @@ qk_rmsnorm_jvp_bwd_kernel(const RmsBwdSide<T> q, const RmsBwdSide<T> k, int H, i
     }
 }
 
-// dg[side][j] = sum over the blocks' partial rows, in block order.
-__global__ void __launch_bounds__(128)
+// dg[side][j] = sum over the blocks' partial rows in a fixed order: eight interleaved partial sums per column
+// (thread t adds the rows b = t / 128, t / 128 + 8, ...), then those eight in order.
+__global__ void __launch_bounds__(1024)
 qk_rmsnorm_dg_reduce_kernel(const float* __restrict__ partial_q, const float* __restrict__ partial_k, float* __restrict__ dg_q,
                             float* __restrict__ dg_k, int nblocks, int d) {
+    __shared__ float acc8[8][128];
     const float* part = blockIdx.x == 0 ? partial_q : partial_k;
     float* out = blockIdx.x == 0 ? dg_q : dg_k;
-    for (int j = threadIdx.x; j < d; j += blockDim.x) {
-        float acc = 0.f;
-        for (int b = 0; b < nblocks; ++b) acc += part[(size_t)b * d + j];
-        out[j] = acc;
+    const int j = threadIdx.x & 127, lane8 = threadIdx.x >> 7;
+    float acc = 0.f;
+    if (j < d)
+        for (int b = lane8; b < nblocks; b += 8) acc += part[(size_t)b * d + j];
+    acc8[lane8][j] = acc;
+    __syncthreads();
+    if (lane8 == 0 && j < d) {
+        float total = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) total += acc8[k][j];
+        out[j] = total;
     }
 }
 

@@ -187,7 +187,7 @@ __device__ __forceinline__ void dot_chunk(const uint4& a, const uint4& b, float&
     }
 }
 
-// `gs` = lanes per row (power of two, >= chunks per row `cpr`); rows_per_warp = 32 / gs.
+// `gs` = lanes per row = chunks per row `cpr`; rows per warp = 32 / gs (the lanes left over idle).
 template <typename T>
 __global__ void __launch_bounds__(ROWSUM_THREADS)
 bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* __restrict__ O,
@@ -205,7 +205,7 @@ bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* _
 #pragma unroll
     for (int u = 0; u < ROWSUM_UNROLL; ++u) {
         const long long row = row0 + (long long)u * rpw;
-        act[u] = row < rows && c < cpr;
+        act[u] = row < rows && c < cpr && sub < rpw;
         g[u] = h[u] = t[u] = make_uint4(0, 0, 0, 0);  // a null G or Hc (absent cotangent) counts as zeros
         if (act[u]) {
             // the statistics are packed (B, H, M); the tensors have strides (H == 0 marks the packed layout: no division)
@@ -231,11 +231,9 @@ bwd_rowsums_kernel(const T* __restrict__ G, const T* __restrict__ Hc, const T* _
             dot_chunk(g[u], o[u], cc, T());
             dot_chunk(h[u], t[u], cc, T());
         }
-        for (int off = gs >> 1; off > 0; off >>= 1) {
-            s1 += __shfl_xor_sync(0xffffffffu, s1, off);
-            cc += __shfl_xor_sync(0xffffffffu, cc, off);
-        }
-        if (c == 0 && row < rows) { sig1[row] = s1; cvec[row] = cc; lse2[row] = lse[row] * 1.4426950408889634f; }
+        s1 = lane_group_sum(s1, gs, lane);
+        cc = lane_group_sum(cc, gs, lane);
+        if (c == 0 && sub < rpw && row < rows) { sig1[row] = s1; cvec[row] = cc; lse2[row] = lse[row] * 1.4426950408889634f; }
     }
 }
 

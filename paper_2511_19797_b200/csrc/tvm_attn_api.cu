@@ -122,8 +122,7 @@ static int launch_rowsums(const Shape& s, const void* G, const void* Hc, const v
                           float* sig1, float* cvec, float* lse2, cudaStream_t st) {
     const long long rows = s.BH * s.M;
     const int cpr = s.d * (int)sizeof(T) / 16;  // 16-byte chunks per row (d % 8 == 0)
-    int gs = 1;
-    while (gs < cpr) gs <<= 1;
+    const int gs = cpr;                          // lanes per row
     if (gs > 32) return TVM_ATTN_UNSUPPORTED;   // d <= 128 keeps a row within one warp
     const long long rows_per_block = (long long)(ROWSUM_THREADS / 32) * ROWSUM_UNROLL * (32 / gs);
     const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
@@ -401,10 +400,8 @@ __global__ void selftest_timeout_kernel(int* status, unsigned long long limit_ns
 // RMSNorm QK-normalisation prologue
 static int rms_geometry(const Shape& s, int* cpr, int* gs) {
     *cpr = s.d * (s.fp32 ? 4 : 2) / 16;
-    int g = 1;
-    while (g < *cpr) g <<= 1;
-    *gs = g;
-    return g <= 32 ? TVM_ATTN_OK : TVM_ATTN_UNSUPPORTED;
+    *gs = *cpr;   // lanes per row
+    return *gs <= 32 ? TVM_ATTN_OK : TVM_ATTN_UNSUPPORTED;
 }
 
 template <typename T>
@@ -435,7 +432,7 @@ static int rms_bwd(const Shape& s, float eps, const void* Q, const void* tQ, con
     const RmsBwdSide<T> q{(const T*)Q, (const T*)tQ, gQ, (const T*)dQn, (const T*)dtQn, (T*)dQ, (T*)dtQ, pq, s.q, s.BH * s.M};
     const RmsBwdSide<T> k{(const T*)K, (const T*)tK, gK, (const T*)dKn, (const T*)dtKn, (T*)dK, (T*)dtK, pk, s.k, s.BH * s.N};
     qk_rmsnorm_jvp_bwd_kernel<T><<<dim3(RMS_BWD_BLOCKS, 2), RMS_THREADS, 0, st>>>(q, k, s.H, s.d, cpr, gs, eps);
-    qk_rmsnorm_dg_reduce_kernel<<<2, 128, 0, st>>>(pq, pk, dgQ, dgK, RMS_BWD_BLOCKS, s.d);
+    qk_rmsnorm_dg_reduce_kernel<<<2, 1024, 0, st>>>(pq, pk, dgQ, dgK, RMS_BWD_BLOCKS, s.d);
     g_launches += 2;
     return cuda_status(cudaGetLastError());
 }
