@@ -803,16 +803,31 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
             const uint64_t b0 = desc64(l_nlo(l_stage(g), 0, 0), HI_SW128);
             const uint64_t b1 = desc64(l_nlo(l_stage(g), 1, 0), HI_SW128);
             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
-            const bool hasH = !HZ && !(p.absent & ABSENT_HC), hasG = !(p.absent & ABSENT_G);  // B0 = Hc, B1 = G
+            if (!HZ && p.absent == 0) {
+                // both cotangents present: the loop as plain as it can be (one uniform branch outside it; a branch per
+                // MMA inside the unrolled loop costs the issuing warp more than it looks)
 #pragma unroll
-            for (int u = 0; u < BC / 16; ++u) {
-                const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
-                const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
-                if (hasH) {
+                for (int u = 0; u < BC / 16; ++u) {
+                    const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                    const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
+                    ptx::mma_ts_elect(acc0, a0 + 16 * u, b0 + off, idesc_o, acc);   // acc0 += A0 B0
+                    ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc_o, acc);   // acc1 += A1 B0
+                    ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, 1u);    // acc1 += A0 B1
+                }
+            } else if (HZ || (p.absent & ABSENT_HC)) {  // B0 = Hc absent
+#pragma unroll
+                for (int u = 0; u < BC / 16; ++u) {
+                    const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                    ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, (j > 0 || u > 0) ? 1u : 0u);  // acc1 += A0 B1
+                }
+            } else {  // B1 = G absent
+#pragma unroll
+                for (int u = 0; u < BC / 16; ++u) {
+                    const uint64_t off = (uint64_t)((u * 16 * 128) >> 4);
+                    const uint32_t acc = (j > 0 || u > 0) ? 1u : 0u;
                     ptx::mma_ts_elect(acc0, a0 + 16 * u, b0 + off, idesc_o, acc);   // acc0 += A0 B0
                     ptx::mma_ts_elect(acc1, a1 + 16 * u, b0 + off, idesc_o, acc);   // acc1 += A1 B0
                 }
-                if (hasG) ptx::mma_ts_elect(acc1, a0 + 16 * u, b1 + off, idesc_o, hasH ? 1u : acc);  // acc1 += A0 B1
             }
             ptx::mma_commit_elect(bar(C::B_LEMPTY + g % SL));
             if (j == T - 1) ptx::mma_commit_elect(bar(C::B_FINAL));
@@ -953,14 +968,20 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                             for (int u = 0; u < BC / 16; ++u) {
                                 const uint32_t off = (uint32_t)((u * 16 * 128) >> 4);
                                 // with Hc absent W is exactly zero (D = 0 from zero operands, Sigma1 = 0): its MMAs are skipped
-                                if (u == 0 && j == 0) {
-                                    if (hasW) ptx::mma_ts_p<0>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
-                                    ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                // (one uniform branch around the three-MMA body, none inside it)
+                                if (hasW) {
+                                    if (u == 0 && j == 0) {
+                                        ptx::mma_ts_p<0>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
+                                        ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    } else {
+                                        ptx::mma_ts_p<1>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
+                                        ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    }
+                                    ptx::mma_ts_p<1>(el, acc1, dD + 16 * u, b1 + off, HI_SW, idesc_o);
                                 } else {
-                                    if (hasW) ptx::mma_ts_p<1>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
-                                    ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    if (u == 0 && j == 0) ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
+                                    else ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
                                 }
-                                if (hasW) ptx::mma_ts_p<1>(el, acc1, dD + 16 * u, b1 + off, HI_SW, idesc_o);
                             }
                             ptx::mma_commit_p(el, bar(C::B_LEMPTY + g % SL));
                             if (j == T - 1) ptx::mma_commit_p(el, bar(C::B_FINAL));
