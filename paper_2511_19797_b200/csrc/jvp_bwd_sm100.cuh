@@ -964,12 +964,12 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                             const uint32_t b0 = l_nlo(l_stage(g), 0, 0), b1 = l_nlo(l_stage(g), 1, 0);  // MN-major B
                             const bool hasW = !HZ && !(p.absent & ABSENT_HC);
                             const uint32_t acc0 = tb + C::COL_ACC0, acc1 = tb + C::COL_ACC1;
+                            // with Hc absent W is exactly zero (D = 0 from zero operands, Sigma1 = 0): its MMAs are skipped.
+                            // One uniform branch around the unrolled loops, none inside them.
+                            if (hasW) {
 #pragma unroll
-                            for (int u = 0; u < BC / 16; ++u) {
-                                const uint32_t off = (uint32_t)((u * 16 * 128) >> 4);
-                                // with Hc absent W is exactly zero (D = 0 from zero operands, Sigma1 = 0): its MMAs are skipped
-                                // (one uniform branch around the three-MMA body, none inside it)
-                                if (hasW) {
+                                for (int u = 0; u < BC / 16; ++u) {
+                                    const uint32_t off = (uint32_t)((u * 16 * 128) >> 4);
                                     if (u == 0 && j == 0) {
                                         ptx::mma_ts_p<0>(el, acc0, dD + 16 * u, b0 + off, HI_SW, idesc_o);
                                         ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
@@ -978,7 +978,11 @@ jvp_bwd_kernel(const __grid_constant__ CUtensorMap tm_s0, const __grid_constant_
                                         ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
                                     }
                                     ptx::mma_ts_p<1>(el, acc1, dD + 16 * u, b1 + off, HI_SW, idesc_o);
-                                } else {
+                                }
+                            } else {
+#pragma unroll
+                                for (int u = 0; u < BC / 16; ++u) {
+                                    const uint32_t off = (uint32_t)((u * 16 * 128) >> 4);
                                     if (u == 0 && j == 0) ptx::mma_ts_p<0>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
                                     else ptx::mma_ts_p<1>(el, acc1, dX + 16 * u, b0 + off, HI_SW, idesc_o);
                                 }
