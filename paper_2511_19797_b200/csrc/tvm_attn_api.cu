@@ -20,6 +20,21 @@
 namespace tvm_attn {
 
 static std::atomic<uint64_t> g_launches{0};
+
+// Number of SMs of the current device (a fact of the hardware: looked up once per device index); <= 0 on error.
+static int device_sm_count() {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return -1;
+    if (dev < 64) {
+        const int v = cached[dev].load(std::memory_order_relaxed);
+        if (v > 0) return v;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return -1;
+    if (dev < 64) cached[dev].store(sms, std::memory_order_relaxed);
+    return sms;
+}
 __device__ int g_status_word = 0;  // raised by a tensor-core kernel whose bounded wait ran out
 
 // Optional per-kernel timing: events recorded around each launch of the most recent call.  While it is
@@ -263,9 +278,8 @@ static int launch_fwd(const Shape& s, const void* const strm[4], const FwdParams
     // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
     // items go round-robin over them
     const long long items = s.BH * ((s.M + FWD_ROWS - 1) / FWD_ROWS);
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-        return TVM_ATTN_CUDA_ERROR;
+    const int sms = device_sm_count();
+    if (sms <= 0) return TVM_ATTN_CUDA_ERROR;
     const long long grid = items < sms ? items : sms;
     g_prof.before(st);
     kern<<<(unsigned)grid, FWD_THREADS, C::SMEM_BYTES, st>>>(m[0], m[1], m[2], m[3], prm);
@@ -302,9 +316,8 @@ static int launch_bwd_pass(const Shape& s, const void* const own[4], const void*
     // one CTA per SM (each needs the whole tensor memory and most of the shared memory of one); the work
     // items go round-robin over them
     const long long items = s.BH * ((prm.o.rows + BWD_ROWS - 1) / BWD_ROWS);
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-        return TVM_ATTN_CUDA_ERROR;
+    const int sms = device_sm_count();
+    if (sms <= 0) return TVM_ATTN_CUDA_ERROR;
     const long long grid = items < sms ? items : sms;
     g_prof.before(st);
     {
