@@ -103,7 +103,10 @@ struct BwdCfg {
     static constexpr int XS0 = NPAIR == 2 ? 0 : 2;  // p.own[XS0], p.own[XS0 + 1] -> shared memory (two-pair passes)
     static constexpr int EST_BYTES = BC * 128 + (NA - 1) * BC * 32;  // one E-ring tile
     static constexpr int LST_BYTES = NA * BC * 128;                  // one L-ring tile
-    static constexpr int SE = NPAIR == 1 ? 4 : (NA == 1 ? 4 : 3);
+    // Ring depths.  The E ring of DK / DQ (second-pair operands, released right after that pair) is kept shallow: two
+    // stages at head dims above 64 measured 2 to 5 % faster than three (and one or a two-stage L ring far slower);
+    // at head dims up to 64, three stages in DK and four in DQ.
+    static constexpr int SE = NPAIR == 1 ? 4 : (NA == 1 ? (MODE == BWD_DK ? 3 : 4) : 2);
     static constexpr int SL = NA == 1 ? 4 : 3;
     static constexpr int TILE_BYTES = NOWN_SMEM * OWN_BYTES + SE * 2 * EST_BYTES + SL * 2 * LST_BYTES;
     static constexpr int FULL_COUNT = NA;                  // TMA issuer (+ the warp copying columns >= 64)
