@@ -311,14 +311,47 @@ def main():
     host_out = {k: torch.empty(shape, dtype=torch.bfloat16).pin_memory() for k in out_names}
     host_stats = {k: torch.empty(shape[:3], dtype=torch.float32).pin_memory() for k in ("lse", "mu")}
 
+    # The batch is cut into chunks (heads are independent) and the three legs run on three streams: while chunk c is
+    # computed, chunk c + 1 comes in and chunk c - 1 goes out.  Events order the legs within a step and across steps
+    # (a chunk's device buffers are rewritten by the next step).
+    n_chunks = 4 if wl.B % 4 == 0 else 1
+    cb = wl.B // n_chunks
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    ev_in = [torch.cuda.Event() for _ in range(n_chunks)]
+    ev_comp = [torch.cuda.Event() for _ in range(n_chunks)]
+    ev_out = [torch.cuda.Event() for _ in range(n_chunks)]
+    ws_c = torch.empty(binding.tvm_attn_jvp_workspace_bytes(cb, wl.H, wl.N, wl.d), dtype=torch.uint8, device=dev)
+    started = [False]
+
     def e2e_step():
-        for k in in_names:
-            x[k].copy_(host[k], non_blocking=True)
-        step()
-        for k, t in zip(out_names, (O, tO) + grads):
-            host_out[k].copy_(t, non_blocking=True)
-        host_stats["lse"].copy_(lse, non_blocking=True)
-        host_stats["mu"].copy_(mu, non_blocking=True)
+        comp = torch.cuda.current_stream()
+        for c in range(n_chunks):
+            sl = slice(c * cb, (c + 1) * cb)
+            if started[0]:
+                s_in.wait_event(ev_comp[c])     # the step before has consumed this chunk's inputs
+            with torch.cuda.stream(s_in):
+                for k in in_names:
+                    x[k][sl].copy_(host[k][sl], non_blocking=True)
+                ev_in[c].record(s_in)
+            comp.wait_event(ev_in[c])
+            if started[0]:
+                comp.wait_event(ev_out[c])      # the step before has copied this chunk's results out
+            binding.tvm_attn_jvp_fwd(x["Q"][sl], x["K"][sl], x["V"][sl], x["tQ"][sl], x["tK"][sl], x["tV"][sl],
+                                     out=(O[sl], tO[sl], lse[sl], mu[sl]))
+            g = tuple(t[sl] for t in grads)
+            binding.tvm_attn_jvp_bwd(x["Q"][sl], x["K"][sl], x["V"][sl], x["tQ"][sl], x["tK"][sl], x["tV"][sl], O[sl], tO[sl],
+                                     lse[sl], mu[sl], x["dO"][sl], None if detach else x["dtO"][sl],
+                                     out=(g[:3] + (None, None, None)) if detach else g, workspace=ws_c)
+            ev_comp[c].record(comp)
+            s_out.wait_event(ev_comp[c])
+            with torch.cuda.stream(s_out):
+                for k, t in zip(out_names, (O, tO) + grads):
+                    host_out[k][sl].copy_(t[sl], non_blocking=True)
+                host_stats["lse"][sl].copy_(lse[sl], non_blocking=True)
+                host_stats["mu"][sl].copy_(mu[sl], non_blocking=True)
+                ev_out[c].record(s_out)
+        comp.wait_event(ev_out[n_chunks - 1])   # the step ends when its last results are on the host
+        started[0] = True
 
     if args.e2e_steps > 0:
         e2e_step()
@@ -427,7 +460,8 @@ def main():
                      "step": {"tensor_frac": step_tensor_frac, "hbm_frac": step_hbm_frac, "bytes": step_bytes}},
         "e2e": None if ms_e2e is None else {
             "value": world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
-            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "pipeline": "%d batch chunks; copy-in, compute and copy-out on three streams" % n_chunks},
         "gpu_launches": launches,
         "clocks": clocks,
     }
