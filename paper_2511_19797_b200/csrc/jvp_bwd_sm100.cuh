@@ -382,8 +382,8 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         if (ok) ok = ptx::mbar_wait_warp(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
         if (ok) {
             ptx::tc_fence_after_sync();
-            __nv_bfloat16* p0 = p.out0 + ooff;
-            __nv_bfloat16* p1 = p.out1 + ooff;
+            // DK: lane pairs write the two rows of the pair one after the other, each as complete 32-byte sectors
+            [[maybe_unused]] const bool ok_even = row0 + (row & ~1) < p.o.rows, ok_odd = row0 + (row | 1) < p.o.rows;
             for (int ch = slot; ch < KS; ch += 4) {
                 uint32_t x0[16], x1[16];
                 ptx::tmem_ld16(lane_addr + C::COL_ACC0 + 16 * ch, x0);
@@ -395,12 +395,19 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                     q0[c >> 1] = ptx::pack_bf16(__uint_as_float(x0[c]) * p.out_scale, __uint_as_float(x0[c + 1]) * p.out_scale);
                     q1[c >> 1] = ptx::pack_bf16(__uint_as_float(x1[c]) * p.out_scale, __uint_as_float(x1[c + 1]) * p.out_scale);
                 }
-                if (row_valid) {
-                    *reinterpret_cast<uint4*>(p1 + 16 * ch) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
-                    if (16 * ch + 8 < p.d) *reinterpret_cast<uint4*>(p1 + 16 * ch + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
-                    if (p.out0) {  // null with Hc absent: acc0 was never written and its gradient is zero
-                        *reinterpret_cast<uint4*>(p0 + 16 * ch) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
-                        if (16 * ch + 8 < p.d) *reinterpret_cast<uint4*>(p0 + 16 * ch + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
+                const bool has_hi = 16 * ch + 8 < p.d;
+                __nv_bfloat16* p0 = p.out0 + ooff + 16 * ch;  // out0 is null with Hc absent: acc0 was never written, its gradient is zero
+                __nv_bfloat16* p1 = p.out1 + ooff + 16 * ch;
+                if constexpr (MODE == BWD_DK) {
+                    // (measured: DK 2 to 6 % faster this way, DQ the same, DV 2 % slower)
+                    store_row_pairs(p1, p.o.rs, lane, ok_even, ok_odd, has_hi, make_uint4(q1[0], q1[1], q1[2], q1[3]), make_uint4(q1[4], q1[5], q1[6], q1[7]));
+                    if (p.out0) store_row_pairs(p0, p.o.rs, lane, ok_even, ok_odd, has_hi, make_uint4(q0[0], q0[1], q0[2], q0[3]), make_uint4(q0[4], q0[5], q0[6], q0[7]));
+                } else if (row_valid) {
+                    *reinterpret_cast<uint4*>(p1) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
+                    if (has_hi) *reinterpret_cast<uint4*>(p1 + 8) = make_uint4(q1[4], q1[5], q1[6], q1[7]);
+                    if (p.out0) {
+                        *reinterpret_cast<uint4*>(p0) = make_uint4(q0[0], q0[1], q0[2], q0[3]);
+                        if (has_hi) *reinterpret_cast<uint4*>(p0 + 8) = make_uint4(q0[4], q0[5], q0[6], q0[7]);
                     }
                 }
             }
