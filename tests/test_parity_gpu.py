@@ -94,8 +94,10 @@ def test_explicit_scale_is_honoured():
     assert_within(errs, BF16_FWD, BF16_BWD, BF16_STATS)
 
 
-def test_runs_are_bit_reproducible_and_respect_buffer_bounds():
-    wl = inputs.custom(2, 2, 200, 72, seed=9)
+@pytest.mark.parametrize("N,d", [(200, 72), (129, 72), (65, 64)])
+def test_runs_are_bit_reproducible_and_respect_buffer_bounds(N, d):
+    # (an odd number of rows: the last row has no partner in the pass that writes its outputs by lane pairs)
+    wl = inputs.custom(2, 2, N, d, seed=9)
     x = {k: v.to(torch.bfloat16).cuda() for k, v in inputs.make_inputs(wl).items()}
     n = x["Q"].numel()
 
