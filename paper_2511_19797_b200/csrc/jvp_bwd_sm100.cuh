@@ -208,6 +208,22 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
     bool ok = true;
     int it = 0;  // items done by this CTA
     if ((int)blockIdx.x < items) stage_x(blockIdx.x, 0);
+    // DQ: the statistics of this thread's row in the next item, loaded before the epilogue's stores go out (behind
+    // them the loads would wait in the same queue)
+    [[maybe_unused]] float n_lse2 = CUDART_INF_F, n_mu = 0.f, n_s1 = 0.f, n_cv = 0.f;
+    [[maybe_unused]] auto load_stats = [&](int item_) {
+        const int bh_ = item_ / row_tiles;
+        const int row0_ = (item_ - bh_ * row_tiles) * BWD_ROWS;
+        n_lse2 = CUDART_INF_F; n_mu = 0.f; n_s1 = 0.f; n_cv = 0.f;
+        if (row0_ + row < p.o.rows) {
+            const size_t grow_ = (size_t)bh_ * p.o.rows + row0_ + row;
+            n_lse2 = p.lse2[grow_];
+            n_mu = p.mu[grow_];
+            n_s1 = p.sig1[grow_];
+            n_cv = p.cvec[grow_];
+        }
+    };
+    if (MODE == BWD_DQ && (int)blockIdx.x < items) load_stats(blockIdx.x);
     for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++it) {
         const int g0 = it * T;  // tiles this CTA has streamed before this item: rings and barrier phases run on
         const int bh = item / row_tiles;
@@ -215,13 +231,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
         const bool row_valid = row0 + row < p.o.rows;
         const size_t grow = (size_t)bh * p.o.rows + row0 + row;   // DQ: this query's slot in the packed statistics
         const size_t ooff = p.o.head_off(bh, p.H) + (size_t)(row0 + row) * (size_t)p.o.rs;
-        float r_lse2 = CUDART_INF_F, r_mu = 0.f, r_s1 = 0.f, r_cv = 0.f;  // per-row statistics (DQ)
-        if (MODE == BWD_DQ && row_valid) {
-            r_lse2 = p.lse2[grow];
-            r_mu = p.mu[grow];
-            r_s1 = p.sig1[grow];
-            r_cv = p.cvec[grow];
-        }
+        const float r_lse2 = n_lse2, r_mu = n_mu, r_s1 = n_s1, r_cv = n_cv;  // per-row statistics (DQ)
         for (int j = NPAIR == 1 ? ((par ^ g0) & 1) : 0; j < T; j += jstep) {
             const int g = g0 + j;
             const int b = NPAIR == 1 ? (g & 1) : 0, sph = NPAIR == 1 ? (g >> 1) & 1 : (g & 1);
@@ -378,6 +388,7 @@ __device__ __forceinline__ void bwd_elementwise(const BwdParams& p, uint32_t tme
                 if (!ptx::mbar_wait_warp(bar(C::B_SFULL + (gl & 1)), (gl >> 1) & 1, abort_flag, BWD_WAIT_LIMIT_NS)) { ok = false; break; }
             }
             stage_x(item + gridDim.x, it + 1);
+            if (MODE == BWD_DQ) load_stats(item + gridDim.x);
         }
         if (ok) ok = ptx::mbar_wait_warp(bar(C::B_FINAL), it & 1, abort_flag, BWD_WAIT_LIMIT_NS);
         if (ok) {
