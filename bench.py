@@ -38,7 +38,7 @@ KERNEL_TENSORS = {"fwd": 8, "bwd_rowsums": 4, "bwd_dv": 8, "bwd_dk": 10, "bwd_dq
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
 # profiles/jvp_fwd_bwd_kernels_dit512.md (that workload only; None for anything else, and None once a kernel
 # has changed since the capture)
-NCU_TRAFFIC_BYTES = {"dit512": {"fwd": 281.1e6, "bwd_dv": 281.7e6, "bwd_dk": 365.9e6, "bwd_dq": 363.8e6}}
+NCU_TRAFFIC_BYTES = {"dit512": {"fwd": 280.0e6, "bwd_dv": 281.5e6, "bwd_dk": 366.3e6, "bwd_dq": 363.7e6}}
 
 
 def load_peaks():
