@@ -14,7 +14,10 @@
  *     allocates, frees or keeps device memory.
  *   - Outputs are fully overwritten, never accumulated into.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
- *     and the call returns without synchronising.
+ *     and the call returns without synchronising.  The forward and backward calls neither allocate
+ *     nor synchronise, so they may be recorded into a CUDA graph by stream capture (make one call
+ *     per device outside capture first: it loads the kernels); tvm_attn_check_status synchronises
+ *     and the timing aid records events, so neither belongs inside a capture.
  *   - Return value: TVM_ATTN_OK or a negative tvm_attn_status.  No exception or abort crosses
  *     this boundary.  Concurrent calls from several host threads on different streams are allowed
  *     (each call with its own workspace); the per-kernel timing aid below is the exception and is to
