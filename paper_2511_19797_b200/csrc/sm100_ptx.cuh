@@ -319,7 +319,7 @@ __device__ __forceinline__ void mma_commit_p(uint32_t el, uint32_t bar) {
 }
 
 // Bounded wait executed by a whole warp; the result is made warp-uniform.  (All lanes poll: letting
-// lane 0 poll alone and broadcasting its verdict measured slower.)
+// lane 0 poll alone and broadcasting the result measured slower.)
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
     const bool ok = mbar_wait(bar, parity, abort_flag, limit_ns);
     return __all_sync(0xffffffffu, ok);
